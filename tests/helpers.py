@@ -1,0 +1,132 @@
+"""Test-side helpers: library softmax tables, exact branch enumeration, closed forms, tie accounting.
+
+Nothing here is used by the product.  The enumeration drives the oracle through every
+branch of the verification rule with exact weights ("branch-midpoint quadrature"): each
+accept uniform is put at the midpoint of its accept region (0, t] or reject region (t, 1)
+and weighted by that region's length, the sampling uniform at the midpoint of each token's
+CDF interval and weighted by the interval's length.
+"""
+from __future__ import annotations
+
+import itertools
+
+import numpy as np
+from scipy.special import softmax as sp_softmax
+
+
+def prob_tables(models, T):
+    """float64 softmax tables [rows_i, V] per model from (float64-convertible) logits [rows_i, V]."""
+    return [sp_softmax(np.asarray(m, dtype=np.float64) / T, axis=-1) for m in models]
+
+
+def level_branches(P, Q, stream, k_l):
+    """All (a, token, weight, accept_uniforms, sampling_uniform) of one level given the incoming stream."""
+    m = min(k_l, len(stream))
+    out = []
+    for a in range(m + 1):
+        w = 1.0
+        ua = [0.5] * k_l
+        ok = True
+        for j in range(a):
+            t = min(1.0, P[j, stream[j]] / Q[j, stream[j]])
+            w *= t
+            ua[j] = t / 2.0
+        if a < m:
+            t = min(1.0, P[a, stream[a]] / Q[a, stream[a]])
+            if t >= 1.0:
+                ok = False
+            else:
+                w *= 1.0 - t
+                ua[a] = (t + 1.0) / 2.0
+            D = np.maximum(P[a] - Q[a], 0.0)
+        else:
+            D = P[m].copy()
+        if not ok or w == 0.0:
+            continue
+        D = D / D.sum()
+        cdf = np.concatenate([[0.0], np.cumsum(D)])
+        for v in range(len(D)):
+            if D[v] <= 0.0:
+                continue
+            out.append((a, v, w * D[v], list(ua), 0.5 * (cdf[v] + cdf[v + 1])))
+    return m, out
+
+
+def enumerate_chain(tables, k, V):
+    """Yield (weight, uniforms [L, kmax+1], draft tokens, expected per-level (m, a, stream)) over all branches."""
+    n = len(tables)
+    L = n - 1
+    kmax = max(k)
+
+    def rec(l, stream, weight, U, trace):
+        if l < 0:
+            yield weight, U, trace
+            return
+        m, branches = level_branches(tables[l], tables[l + 1], stream, k[l])
+        for a, v, w, ua, us in branches:
+            U2 = U.copy()
+            U2[l, :k[l]] = ua
+            U2[l, kmax] = us
+            yield from rec(l - 1, stream[:a] + [v], weight * w, U2, trace + [(l, m, a, stream[:a] + [v])])
+
+    Qb = tables[n - 1]
+    for draft in itertools.product(range(V), repeat=k[L - 1]):
+        w = 1.0
+        for j, x in enumerate(draft):
+            w *= Qb[j, x]
+        U = np.full((L, kmax + 1), 0.5)
+        for weight, U2, trace in rec(L - 1, list(draft), w, U, []):
+            yield weight, U2, list(draft), trace
+
+
+def expected_accept_len_bottom(P, Q, m):
+    """E[a] = sum_j prod_{i<=j} alpha_i with alpha_i = sum_v min(P_i, Q_i): the bottom level's closed form.
+
+    With a constant alpha this is alpha (1 - alpha^m) / (1 - alpha); counting the replacement/bonus
+    token as well gives (1 - alpha^(m+1)) / (1 - alpha), the capped-geometric mean in the proof of
+    Theorem 3.3 with n = m + 1 and continuation probability alpha.
+    """
+    alpha = np.minimum(P[:m], Q[:m]).sum(axis=-1)
+    return float(np.cumprod(alpha).sum())
+
+
+def expected_accept_len_second(P1, P2, Q3, k1, k2):
+    """E[a] of the level above the bottom one (three consecutive models M_1, M_2, M_3 = drafter).
+
+    Position i < j must carry a draft token accepted by both levels, probability
+    gamma_i = sum_v min(Q3_i, P2_i)(v) min(1, P1_i(v) / P2_i(v)); the token at position j then has
+    law P2_j, so it passes with alpha_j = sum_v min(P1_j, P2_j).  j runs to min(k1, k2 + 1).
+    """
+    J = min(k1, k2 + 1)
+    total, surv = 0.0, 1.0
+    for j in range(J):
+        alpha = np.minimum(P1[j], P2[j]).sum()
+        total += surv * alpha
+        if j < k2:
+            ratio = np.minimum(1.0, P1[j] / P2[j])
+            surv *= (np.minimum(Q3[j], P2[j]) * ratio).sum()
+    return float(total)
+
+
+TIE_BAND = 1e-6
+
+
+def compare_level(gpu_a, gpu_next, ora_a, ora_next, accept_margin, sample_info, band=TIE_BAND):
+    """Classify one (level, sequence) result against the oracle.
+
+    Returns "exact", "tie_accept" (accept decisions differ at a position whose uniform lies within
+    `band` of min(1, P/Q)), "tie_sample" (same accepted length, GPU token is the neighbouring
+    positive-mass token and the sampling uniform lies within `band`, in normalised CDF units, of
+    the edge between them) or "mismatch".
+    """
+    if gpu_a == ora_a and gpu_next == ora_next:
+        return "exact"
+    if gpu_a != ora_a:
+        j = min(gpu_a, ora_a)
+        if 0 <= j < len(accept_margin) and np.isfinite(accept_margin[j]) and accept_margin[j] <= band:
+            return "tie_accept"
+        return "mismatch"
+    margin, _, prev, succ = sample_info
+    if margin <= band and gpu_next in (int(prev), int(succ)) and gpu_next >= 0:
+        return "tie_sample"
+    return "mismatch"
