@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the chained verification step (libpolyspec) on synthetic logits.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2|cfg1|cfg4] [--impl reference]
+
+One step = one pass of the whole hot path (row statistics over every logits row of every model,
+then accept tests / first rejection / replacement-or-bonus sampling / hand-off for every level)
+over one batch that is already resident in HBM.  The default workload is the largest logits-path
+configuration, the four-level chain (B=256 per GPU, V=152064, bf16, k=(10,6,4) bottom-up, 2.57 GB of
+logits per call -- larger than L2, so nothing is served from cache between steps).
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle as it stands on the host
+cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2510_26527_b200 import synth  # noqa: E402
+
+METRIC = "verified_draft_tokens_per_s"
+UNIT = "tokens/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-statistics kernel, from the ncu
+# capture summarised under profiles/ (bytes per logits byte processed, measured on a smaller case of
+# the same kernel and scaled by the bytes one launch processes).  None until a capture exists.
+STATS_TRAFFIC_PER_LOGIT_BYTE = None
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return {"hbm_gbs": float(pk["hbm_gbs"]), "bf16_tflops": float(pk["bf16_tflops"]),
+                "bf16_tflops_sustained": float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+def chain_spec(name: str, sigma: float):
+    return synth.config(name, sigma=sigma)
+
+
+def verified_tokens(block_len) -> int:
+    return int(block_len.clamp(min=0).sum().item())
+
+
+# ----------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(spec, seed, n_seq, device):
+    """The first n_seq sequences of the recipe (same V, rows, dtype), as CPU tensors."""
+    d = synth.make_chain(synth.scaled(spec, B=n_seq), seed=seed, device=device)
+    return {"models": [m.cpu() for m in d["models"]], "k": d["k"], "draft_tokens": d["draft_tokens"].cpu(),
+            "uniforms": d["uniforms"].cpu(), "temperature": d["temperature"]}
+
+
+def oracle_time(sample, threads):
+    from oracle import oracle as orc
+    t0 = time.perf_counter()
+    out = orc.verify_chain(sample["models"], sample["k"], sample["draft_tokens"], sample["uniforms"],
+                           sample["temperature"], threads=threads)
+    dt = time.perf_counter() - t0
+    return int(out["block_len"].clip(min=0).sum()), dt
+
+
+def cpu_baseline(data, spec, target_seconds=12.0):
+    """The oracle, as it stands, on the first sequences of the resident batch: about target_seconds of CPU work."""
+    from oracle import oracle as orc
+    orc.build()
+    cores = os.cpu_count() or 1
+    B = spec.B
+
+    def take(n):
+        return {"models": [m[:n].cpu() for m in data["models"]], "k": data["k"],
+                "draft_tokens": data["draft_tokens"][:n].cpu(), "uniforms": data["uniforms"][:, :n].cpu().contiguous(),
+                "temperature": data["temperature"]}
+    n0 = min(B, cores)
+    tok0, t0 = oracle_time(take(n0), cores)
+    n = int(min(B, max(n0, n0 * target_seconds / max(t0, 1e-3))))
+    n = max(cores, n // cores * cores) if n >= cores else n
+    n = min(n, B)
+    tok, t = oracle_time(take(n), cores)
+    return {"value": tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {B} sequences of the same batch, {tok} verified tokens in {t:.2f} s, "
+                      f"{cores} threads (one sequence per thread)"}
+
+
+def run_reference(args, spec):
+    """--impl reference: the CPU oracle on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as orc
+    orc.build()
+    cores = os.cpu_count() or 1
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    n_seq = min(spec.B, 8 * cores)
+    sample = oracle_sample(spec, seed=args.seed, n_seq=n_seq, device=dev)
+    for _ in range(args.warmup):
+        oracle_time(sample, cores)
+    tokens, elapsed = 0, 0.0
+    for _ in range(args.steps):
+        tok, dt = oracle_time(sample, cores)
+        tokens += tok
+        elapsed += dt
+    value = tokens / elapsed
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * elapsed / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args, spec), "sample": f"{n_seq} sequences per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{n_seq} of {spec.B} sequences of the recipe per step, {args.steps} steps"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_name(args, spec):
+    k_bottom_up = tuple(reversed(spec.k))
+    extra = f", inter-level sigma {args.sigma}" if spec.name == "cfg5" else ""
+    return (f"{spec.name}: {spec.n_models}-level chain, B={spec.B} per GPU, V={spec.V}, "
+            f"{'bf16' if spec.dtype == torch.bfloat16 else 'fp32'} logits, k={k_bottom_up} bottom-up, "
+            f"T={spec.temperature}{extra}")
+
+
+# ----------------------------------------------------------------------------------------- GPU arm
+def run_gpu(args, spec):
+    from paper_2510_26527_b200 import binding, buildlib
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: libpolyspec has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        buildlib.build()
+    if world > 1:
+        dist.barrier()
+    binding.load_library()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # sequences are independent: each rank verifies its own batch, no data-path collective
+    data = synth.make_chain(spec, seed=args.seed, device=dev, batch_offset=rank * spec.B)
+    call = binding.ChainCall(data["models"], data["k"], data["draft_tokens"], data["uniforms"], data["temperature"])
+    logits_bytes = spec.logits_bytes()
+
+    for _ in range(max(args.warmup, 3)):
+        call.launch()
+    torch.cuda.synchronize()
+    tokens_per_step = verified_tokens(call.out["block_len"])
+    emitted_per_step = int(call.out["out_len"][0].sum().item())
+    assert int(call.device_status.item()) == 0
+
+    # ---- device-timed region: K steps, each = row_stats + walk (exactly polyspec_verify_chain), with an
+    # event between the two halves so the dominant kernel's share is measured live
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        call.row_stats()
+        ev[i][1].record()
+        call.walk()
+        ev[i][2].record()
+    stop.record()
+    barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    clocks = sampler.stop() if rank == 0 else None
+    stats_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    walk_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+
+    # ---- end to end: the host-buffer entry point, H2D of every input and D2H of every output inside the region
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_models = [m.cpu().pin_memory() for m in data["models"]]
+    host_tok, host_u = data["draft_tokens"].cpu().pin_memory(), data["uniforms"].cpu().pin_memory()
+    rows = [int(m.shape[1]) for m in host_models]
+    ws_bytes = binding.polyspec_verify_chain_host_workspace(data["k"], rows, spec.B, spec.V, call.dt)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    host_out = binding.chain_outputs(spec.n_models - 1, spec.B, spec.kmax, "cpu", pin=True)
+    h2d = sum(m.numel() * m.element_size() for m in host_models) + host_tok.numel() * 4 + host_u.numel() * 4
+    d2h = sum(v.numel() * 4 for v in host_out.values()) + 4
+    binding.polyspec_verify_chain_host(host_models, data["k"], host_tok, host_u, data["temperature"], ws, out=host_out)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        binding.polyspec_verify_chain_host(host_models, data["k"], host_tok, host_u, data["temperature"], ws, out=host_out)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    same = all(bool((host_out[k].to(dev) == call.out[k]).all()) for k in ("accepted_len", "block_len", "out_tokens", "out_len"))
+    del ws, host_models
+
+    # ---- reduce over ranks: max time, summed work
+    t = torch.tensor([elapsed_ms, e2e_ms, stats_ms, walk_ms], device=dev, dtype=torch.float64)
+    w = torch.tensor([tokens_per_step, emitted_per_step], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    elapsed_ms, e2e_ms, stats_ms, walk_ms = (float(x) for x in t.tolist())
+    tokens_all, emitted_all = (float(x) for x in w.tolist())
+
+    base = None
+    if rank == 0 and not args.no_cpu_baseline:
+        base = cpu_baseline(data, spec, target_seconds=args.cpu_seconds)
+
+    if rank == 0:
+        peaks = read_peaks()
+        ms_per_step = elapsed_ms / args.steps
+        value = tokens_all * args.steps / (elapsed_ms * 1e-3)
+        achieved = logits_bytes / (stats_ms * 1e-3) / 1e9
+        traffic = None if STATS_TRAFFIC_PER_LOGIT_BYTE is None else STATS_TRAFFIC_PER_LOGIT_BYTE * logits_bytes
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_name(args, spec), "seed": args.seed,
+                       "l2": f"inputs {logits_bytes / 1e9:.3f} GB per step, larger than the 126 MB L2; no flush needed"
+                             if logits_bytes > 4 * 126e6 else "inputs fit in L2: L2-warm timing",
+                       "parallelism": f"{world} independent replicas, batch sharded, no collective"},
+            "gpu_launches": 2 * args.steps,
+            "emitted_tokens_per_s": emitted_all * args.steps / (elapsed_ms * 1e-3),
+            "whole_step_gbs": logits_bytes * world / (ms_per_step * 1e-3) / 1e9,
+            "whole_step_frac_of_hbm_peak": logits_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "kernel_ms": {"row_stats": stats_ms, "walk": walk_ms},
+            "roofline": {"bound": "hbm", "kernel": "stats_kernel (row statistics, every logit once)",
+                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                         "traffic": traffic, "peak_source": f"of {peaks['source']}",
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "e2e": {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                    "matches_device_path": same},
+            "clocks": clocks,
+        }
+        if base is not None:
+            line["cpu_baseline"] = base
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="polyspec", choices=["polyspec", "reference"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--sigma", type=float, default=1.0, help="inter-level noise of cfg5")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    spec = chain_spec(args.workload, args.sigma)
+    if args.impl == "reference":
+        run_reference(args, spec)
+    else:
+        run_gpu(args, spec)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,181 @@
+/*
+ * polyspec.h -- C ABI of libpolyspec: the chained speculative-sampling verification
+ * step of polybasic speculative decoding, as CUDA kernels for sm_100a.
+ *
+ * Vocabulary of the paper (Section 3.1, Problem Formulation): a chain of models
+ * M_1 (the target) ... M_n (the smallest drafter); p_i(x | x_<=t) is model i's
+ * distribution over the vocabulary at a position; M_n drafts a block of tokens that is
+ * "verified in ascending order by M_{n-1}, ..., M_1"; the acceptance length of a
+ * verifier (Eq. 1) is the number of consecutive block tokens it accepts.  A *level* is
+ * one adjacent pair: verifier M_l checking the token stream handed up by M_{l+1}.
+ *
+ * The rule at a level (Algorithm 1: Verify in the inner loop with a break at the first
+ * failure, then VerifyBlock / SampleOne for the level above; the rule itself is
+ * speculative sampling, Sections 2 and 3.1):
+ *   P_j = softmax(logits_p[j] / T), Q_j = softmax(logits_q[j] / T);
+ *   position j is accepted iff  u_j * Q_j(x_j) <= P_j(x_j)   (u_j <= min(1, P/Q));
+ *   accepted_len = a = number of accepted positions before the first rejection;
+ *   next_token   = inverse CDF at the sampling uniform of
+ *                    normalised max(0, P_{a+1} - Q_{a+1})   if a < block_len (residual)
+ *                    P_{block_len+1}                         if a = block_len (bonus row),
+ *                  in ascending vocabulary order, first v whose running sum exceeds u * total.
+ * The emitted stream (x_1..x_a, next_token) is what the next level up verifies, with
+ * that level's q = this level's verifier rows.
+ *
+ * Conventions for every call
+ *   - All pointers are DEVICE pointers owned by the caller unless a parameter says
+ *     "host".  Logits buffers must be 16-byte aligned and V * sizeof(element) must be a
+ *     multiple of 16.  Row-major, innermost dimension = vocabulary.
+ *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and return; outputs are valid once the stream has synchronised.
+ *   - The library allocates no device memory: the caller passes a workspace of at least
+ *     the size the matching *_workspace call reports, 256-byte aligned.  Concurrent calls
+ *     need distinct workspaces.
+ *   - Uniforms are caller-supplied floats in the open interval (0, 1); the library draws
+ *     no random numbers.  Outputs are a pure function of the inputs.
+ *   - Problems visible on the host (NULL pointers, sizes out of range, misalignment,
+ *     temperature <= 0 or not finite, workspace too small) return an error status and
+ *     launch nothing.  Problems only visible on the device (a token outside [0, V), a row
+ *     holding NaN / +inf or no finite logit) never trap: the affected sequence gets
+ *     accepted_len = next_token = -1 (and -1 in every later level of a chain) and
+ *     *device_status is set to POLYSPEC_ERR_BAD_INPUT_ON_DEVICE.
+ */
+#ifndef POLYSPEC_H
+#define POLYSPEC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define POLYSPEC_MAX_K       32   /* largest block a level may verify */
+#define POLYSPEC_MAX_MODELS   8   /* largest chain */
+
+typedef enum {
+    POLYSPEC_OK = 0,
+    POLYSPEC_ERR_INVALID_ARG = 1,
+    POLYSPEC_ERR_UNSUPPORTED = 2,
+    POLYSPEC_ERR_WORKSPACE = 3,
+    POLYSPEC_ERR_CUDA = 4,
+    POLYSPEC_ERR_TIMEOUT = 5,
+    POLYSPEC_ERR_BAD_INPUT_ON_DEVICE = 6
+} polyspec_status;
+
+typedef enum { POLYSPEC_F32 = 0, POLYSPEC_BF16 = 1 } polyspec_dtype;
+
+/* Static strings; never NULL. */
+const char* polyspec_status_string(polyspec_status s);
+/* major * 10000 + minor * 100 + patch */
+int polyspec_version(void);
+
+/*
+ * polyspec_verify_level -- one adjacent pair (verifier p, drafter-side q) over a batch of
+ * independent sequences: Algorithm 1's Verify loop plus the replacement / bonus token.
+ *
+ *   logits_p      [B, k+1, V]  verifier logits; row j scores block position j, row k is the bonus row
+ *   logits_q      [B, k,   V]  logits of the distribution the block tokens were drawn from
+ *   draft_tokens  [B, k]       block tokens, each in [0, V)
+ *   uniforms      [B, k+1]     [b, j<k] accept uniform of position j; [b, k] the sampling uniform
+ *   block_len     [B] or NULL  tokens actually presented per sequence (0..k); NULL means k
+ *   accepted_len  out [B]      0..block_len[b]
+ *   next_token    out [B]      residual sample if accepted_len < block_len, else bonus sample
+ *   p_at_draft, q_at_draft  out [B, k] or NULL: P_j(x_j), Q_j(x_j) for j < block_len, 0 elsewhere
+ *   device_status out [1] or NULL: left untouched when all is well (zero it before the call)
+ */
+polyspec_status polyspec_verify_level_workspace(int B, int k, int V, polyspec_dtype dt, size_t* bytes /* host out */);
+polyspec_status polyspec_verify_level(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
+    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * polyspec_verify_chain -- n models, n-1 levels, verified bottom-up in one call
+ * (Section 3.1; Algorithm 1 is the n = 3 case).  Level index l = 0 .. n-2: verifier is
+ * models[l]; models[0] = M_1 (target), models[n-1] = M_n (bottom drafter).
+ *
+ *   models        host array [n_models]: device pointer to [B, rows, V] logits and its row
+ *                 count; rows >= k[l] + 1 for l < n-1, rows >= k[n-2] for the drafter
+ *   k             host [n_models-1]; k[l] = largest block level l verifies; k[n-2] = draft length
+ *   draft_tokens  [B, k[n-2]]
+ *   uniforms      [n_models-1, B, kmax+1], kmax = max k[l]; level l uses [l, b, j < k[l]] for
+ *                 its accept tests and [l, b, kmax] as its sampling uniform
+ *   Level l verifies the first min(k[l], out_len[l+1]) tokens of the stream emitted by
+ *   level l+1 against q = models[l+1]'s rows.
+ *   accepted_len, block_len, out_len   out [n_models-1, B]; out_len = accepted_len + 1
+ *   out_tokens    out [n_models-1, B, kmax+1]: stream emitted by each level, -1 past out_len;
+ *                 level 0's stream is the committed output
+ */
+typedef struct {
+    const void* logits;   /* device pointer, [B, rows, V] */
+    int rows;
+} polyspec_model_logits;
+
+polyspec_status polyspec_verify_chain_workspace(int n_models, const int* k /* host */, const int* rows /* host [n_models] */,
+                                                int B, int V, polyspec_dtype dt, size_t* bytes /* host out */);
+polyspec_status polyspec_verify_chain(
+    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */,
+    const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The two halves of polyspec_verify_chain, for callers that want to time or overlap them:
+ *   polyspec_chain_row_stats  the temperature-softmax normaliser of every row of every model
+ *                             (the single pass over all logits; Section 3.1's p_i over the
+ *                             vocabulary) written to the workspace;
+ *   polyspec_chain_walk       everything after it (Algorithm 1's accept loop, first rejection,
+ *                             replacement / bonus token, hand-off between levels), reading the
+ *                             workspace the first half filled on the same stream.
+ * Calling one after the other with the same arguments is exactly polyspec_verify_chain.
+ */
+polyspec_status polyspec_chain_row_stats(
+    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */, int B, int V,
+    polyspec_dtype dt, float temperature, void* workspace, size_t workspace_bytes, void* cuda_stream);
+polyspec_status polyspec_chain_walk(
+    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */,
+    const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * polyspec_verify_chain_host -- the same call for a caller whose buffers live in HOST
+ * memory (pinned memory makes the copies asynchronous): logits, draft tokens and
+ * uniforms are copied to a device staging area inside the caller's workspace, the chain
+ * runs, and the four outputs are copied back, all on `cuda_stream`.  Every data pointer
+ * here is a host pointer with the layouts above; `host_status` (host, [1], may be NULL)
+ * receives the device status word.  Outputs are valid after the stream synchronises.
+ */
+polyspec_status polyspec_verify_chain_host_workspace(int n_models, const int* k, const int* rows, int B, int V,
+                                                     polyspec_dtype dt, size_t* bytes /* host out */);
+polyspec_status polyspec_verify_chain_host(
+    const polyspec_model_logits* models_host /* host array of HOST logits pointers */, int n_models, const int* k,
+    const int32_t* draft_tokens_host, const float* uniforms_host, int B, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len_host, int32_t* block_len_host, int32_t* out_tokens_host, int32_t* out_len_host,
+    int32_t* host_status, void* workspace /* device */, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * polyspec_verify_from_hidden -- polyspec_verify_level with the LM-head projection fused
+ * in front (the last op of the model forwards in Algorithm 1, "p_{1:K} <- M_2(...)" and
+ * "v <- M_1(...)"): logits[b, j, v] = sum_d hidden[b, j, d] * W[v, d], bf16 inputs,
+ * fp32 accumulation on the tensor cores; logits are never passed in.
+ *
+ *   hidden_p [B, k+1, d_p] bf16, W_p [V, d_p] bf16 (row-major, d contiguous)
+ *   hidden_q [B, rows_q, d_q] bf16 with rows_q >= k (rows past k-1 are ignored), W_q [V, d_q] bf16
+ *   d_p, d_q multiples of 64; V a multiple of 8; all four buffers 16-byte aligned
+ *   the remaining arguments are those of polyspec_verify_level
+ */
+polyspec_status polyspec_verify_from_hidden_workspace(int B, int k, int V, int d_p, int d_q, size_t* bytes /* host out */);
+polyspec_status polyspec_verify_from_hidden(
+    const void* hidden_p, const void* W_p, const void* hidden_q, const void* W_q, int rows_q,
+    const int32_t* draft_tokens, const float* uniforms, const int32_t* block_len,
+    int B, int k, int V, int d_p, int d_q, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POLYSPEC_H */

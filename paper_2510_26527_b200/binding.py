@@ -1,0 +1,353 @@
+"""Python front end of libpolyspec's C ABI (include/polyspec.h): argument marshalling only.
+
+Each function here has the name and the arguments of the C entry point it calls; torch
+is used for device memory and streams, nothing is computed in Python.  If the CUDA
+library cannot be loaded the functions raise: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpolyspec.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_INPUT_ON_DEVICE = 1, 2, 3, 4, 5, 6
+F32, BF16 = 0, 1
+MAX_K, MAX_MODELS = 32, 8
+
+EXPORTS = (
+    "polyspec_status_string", "polyspec_version",
+    "polyspec_verify_level_workspace", "polyspec_verify_level",
+    "polyspec_verify_chain_workspace", "polyspec_verify_chain",
+    "polyspec_chain_row_stats", "polyspec_chain_walk",
+    "polyspec_verify_chain_host_workspace", "polyspec_verify_chain_host",
+    "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden",
+)
+
+
+class PolyspecError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class ModelLogits(ctypes.Structure):
+    _fields_ = [("logits", ctypes.c_void_p), ("rows", ctypes.c_int)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libpolyspec.so from the package directory; raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_26527_b200.buildlib` "
+                           "(needs nvcc); libpolyspec has no CPU fallback")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+    ci, cf, sz = ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    szp, cip = ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_int)
+    lib.polyspec_status_string.restype = ctypes.c_char_p
+    lib.polyspec_status_string.argtypes = [ci]
+    lib.polyspec_version.restype = ci
+    lib.polyspec_version.argtypes = []
+    lib.polyspec_verify_level_workspace.restype = ci
+    lib.polyspec_verify_level_workspace.argtypes = [ci, ci, ci, ci, szp]
+    lib.polyspec_verify_level.restype = ci
+    lib.polyspec_verify_level.argtypes = [vp, vp, i32p, f32p, i32p, ci, ci, ci, ci, cf,
+                                          i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
+    lib.polyspec_verify_chain_workspace.restype = ci
+    lib.polyspec_verify_chain_workspace.argtypes = [ci, cip, cip, ci, ci, ci, szp]
+    lib.polyspec_verify_chain.restype = ci
+    lib.polyspec_verify_chain.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, i32p, f32p, ci, ci, ci, cf,
+                                          i32p, i32p, i32p, i32p, i32p, vp, sz, vp]
+    lib.polyspec_chain_row_stats.restype = ci
+    lib.polyspec_chain_row_stats.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, vp, sz, vp]
+    lib.polyspec_chain_walk.restype = ci
+    lib.polyspec_chain_walk.argtypes = lib.polyspec_verify_chain.argtypes
+    lib.polyspec_verify_chain_host_workspace.restype = ci
+    lib.polyspec_verify_chain_host_workspace.argtypes = [ci, cip, cip, ci, ci, ci, szp]
+    lib.polyspec_verify_chain_host.restype = ci
+    lib.polyspec_verify_chain_host.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, i32p, f32p, ci, ci, ci, cf,
+                                               i32p, i32p, i32p, i32p, i32p, vp, sz, vp]
+    lib.polyspec_verify_from_hidden_workspace.restype = ci
+    lib.polyspec_verify_from_hidden_workspace.argtypes = [ci, ci, ci, ci, ci, szp]
+    lib.polyspec_verify_from_hidden.restype = ci
+    lib.polyspec_verify_from_hidden.argtypes = [vp, vp, vp, vp, ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf,
+                                                i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().polyspec_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return load_library().polyspec_version()
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(st: int, where: str):
+    if st != OK:
+        raise PolyspecError(st, where)
+
+
+def _dev_check(*tensors):
+    for t in tensors:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("device-pointer arguments must be contiguous CUDA tensors")
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------ verify_level
+def polyspec_verify_level_workspace(B: int, k: int, V: int, dt: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().polyspec_verify_level_workspace(B, k, V, dt, ctypes.byref(n)), "polyspec_verify_level_workspace")
+    return n.value
+
+
+def polyspec_verify_level(logits_p, logits_q, draft_tokens, uniforms, temperature, block_len=None,
+                          want_probs=False, workspace=None, out=None, device_status=None, stream=None):
+    """One adjacent pair over a batch.  logits_p [B,k+1,V], logits_q [B,k,V], draft_tokens [B,k] int32,
+    uniforms [B,k+1] float32; returns device tensors accepted_len [B], next_token [B] (and p_at_draft,
+    q_at_draft [B,k] if want_probs) plus the device status word."""
+    lib = load_library()
+    _dev_check(logits_p, logits_q, draft_tokens, uniforms, block_len)
+    B, rows_p, V = logits_p.shape
+    k = draft_tokens.shape[1]
+    if rows_p != k + 1 or tuple(logits_q.shape) != (B, k, V) or tuple(uniforms.shape) != (B, k + 1):
+        raise ValueError("shapes must be logits_p [B,k+1,V], logits_q [B,k,V], draft_tokens [B,k], uniforms [B,k+1]")
+    if draft_tokens.dtype != torch.int32 or uniforms.dtype != torch.float32 or logits_q.dtype != logits_p.dtype:
+        raise TypeError("draft_tokens int32, uniforms float32, logits_p/logits_q one dtype")
+    dev = logits_p.device
+    dt = _dt(logits_p)
+    if workspace is None:
+        workspace = _workspace(polyspec_verify_level_workspace(B, k, V, dt), dev)
+    if out is None:
+        out = {"accepted_len": torch.empty(B, dtype=torch.int32, device=dev),
+               "next_token": torch.empty(B, dtype=torch.int32, device=dev)}
+        if want_probs:
+            out["p_at_draft"] = torch.empty((B, k), dtype=torch.float32, device=dev)
+            out["q_at_draft"] = torch.empty((B, k), dtype=torch.float32, device=dev)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib.polyspec_verify_level(
+        _ptr(logits_p), _ptr(logits_q), _ptr(draft_tokens), _ptr(uniforms), _ptr(block_len),
+        B, k, V, dt, float(temperature), _ptr(out["accepted_len"]), _ptr(out["next_token"]),
+        _ptr(out.get("p_at_draft")), _ptr(out.get("q_at_draft")), _ptr(device_status),
+        _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "polyspec_verify_level")
+    out["device_status"] = device_status
+    return out
+
+
+# ------------------------------------------------------------------ verify_chain
+def _int_array(vals: Sequence[int]):
+    return (ctypes.c_int * len(vals))(*[int(v) for v in vals])
+
+
+def polyspec_verify_chain_workspace(k: Sequence[int], rows: Sequence[int], B: int, V: int, dt: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().polyspec_verify_chain_workspace(len(rows), _int_array(k), _int_array(rows), B, V, dt, ctypes.byref(n)),
+           "polyspec_verify_chain_workspace")
+    return n.value
+
+
+def chain_outputs(L: int, B: int, kmax: int, device, pin=False) -> dict:
+    kw = {"dtype": torch.int32, "device": device}
+    if pin:
+        kw["pin_memory"] = True
+    return {"accepted_len": torch.empty((L, B), **kw), "block_len": torch.empty((L, B), **kw),
+            "out_tokens": torch.empty((L, B, kmax + 1), **kw), "out_len": torch.empty((L, B), **kw)}
+
+
+def polyspec_verify_chain(models, k, draft_tokens, uniforms, temperature, workspace=None, out=None,
+                          device_status=None, stream=None):
+    """n models (models[0] = M_1 ... models[-1] = M_n, each [B, rows_i, V]), n-1 levels verified bottom-up.
+    k[l] = largest block level l verifies; draft_tokens [B, k[-1]]; uniforms [n-1, B, max(k)+1]."""
+    lib = load_library()
+    _dev_check(*models, draft_tokens, uniforms)
+    n = len(models)
+    L = n - 1
+    B, _, V = models[0].shape
+    dt = _dt(models[0])
+    rows = [int(m.shape[1]) for m in models]
+    kmax = max(int(x) for x in k)
+    if any(m.dtype != models[0].dtype or m.shape[0] != B or m.shape[2] != V for m in models):
+        raise ValueError("all models must share dtype, batch and vocabulary")
+    if tuple(uniforms.shape) != (L, B, kmax + 1) or tuple(draft_tokens.shape) != (B, int(k[-1])):
+        raise ValueError("uniforms must be [n-1, B, max(k)+1] and draft_tokens [B, k[-1]]")
+    if draft_tokens.dtype != torch.int32 or uniforms.dtype != torch.float32:
+        raise TypeError("draft_tokens int32, uniforms float32")
+    dev = models[0].device
+    if workspace is None:
+        workspace = _workspace(polyspec_verify_chain_workspace(k, rows, B, V, dt), dev)
+    if out is None:
+        out = chain_outputs(L, B, kmax, dev)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    arr = (ModelLogits * n)(*[ModelLogits(m.data_ptr(), r) for m, r in zip(models, rows)])
+    st = lib.polyspec_verify_chain(arr, n, _int_array(k), _ptr(draft_tokens), _ptr(uniforms), B, V, dt, float(temperature),
+                                   _ptr(out["accepted_len"]), _ptr(out["block_len"]), _ptr(out["out_tokens"]),
+                                   _ptr(out["out_len"]), _ptr(device_status), _ptr(workspace), workspace.numel(),
+                                   _stream(stream))
+    _check(st, "polyspec_verify_chain")
+    out["device_status"] = device_status
+    return out
+
+
+class ChainCall:
+    """A prepared polyspec_verify_chain call: arguments marshalled once, outputs and workspace allocated once.
+
+    launch() is the single C-ABI call; row_stats() and walk() are its two halves
+    (polyspec_chain_row_stats / polyspec_chain_walk)."""
+
+    def __init__(self, models, k, draft_tokens, uniforms, temperature, stream=None):
+        self.lib = load_library()
+        _dev_check(*models, draft_tokens, uniforms)
+        self.models, self.draft_tokens, self.uniforms = list(models), draft_tokens, uniforms
+        self.n = len(models)
+        self.B, _, self.V = models[0].shape
+        self.dt = _dt(models[0])
+        self.rows = [int(m.shape[1]) for m in models]
+        self.k = [int(x) for x in k]
+        self.kmax = max(self.k)
+        self.temperature = float(temperature)
+        dev = models[0].device
+        self.workspace = _workspace(polyspec_verify_chain_workspace(self.k, self.rows, self.B, self.V, self.dt), dev)
+        self.out = chain_outputs(self.n - 1, self.B, self.kmax, dev)
+        self.device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.out["device_status"] = self.device_status
+        self._arr = (ModelLogits * self.n)(*[ModelLogits(m.data_ptr(), r) for m, r in zip(models, self.rows)])
+        self._k = _int_array(self.k)
+        self.stream = stream
+
+    def _tail(self):
+        o = self.out
+        return (_ptr(o["accepted_len"]), _ptr(o["block_len"]), _ptr(o["out_tokens"]), _ptr(o["out_len"]),
+                _ptr(self.device_status), _ptr(self.workspace), self.workspace.numel(), _stream(self.stream))
+
+    def launch(self):
+        _check(self.lib.polyspec_verify_chain(self._arr, self.n, self._k, _ptr(self.draft_tokens), _ptr(self.uniforms),
+                                              self.B, self.V, self.dt, self.temperature, *self._tail()), "polyspec_verify_chain")
+        return self.out
+
+    def row_stats(self):
+        _check(self.lib.polyspec_chain_row_stats(self._arr, self.n, self._k, self.B, self.V, self.dt, self.temperature,
+                                                 _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)),
+               "polyspec_chain_row_stats")
+
+    def walk(self):
+        _check(self.lib.polyspec_chain_walk(self._arr, self.n, self._k, _ptr(self.draft_tokens), _ptr(self.uniforms),
+                                            self.B, self.V, self.dt, self.temperature, *self._tail()), "polyspec_chain_walk")
+        return self.out
+
+
+def polyspec_verify_chain_host_workspace(k: Sequence[int], rows: Sequence[int], B: int, V: int, dt: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().polyspec_verify_chain_host_workspace(len(rows), _int_array(k), _int_array(rows), B, V, dt, ctypes.byref(n)),
+           "polyspec_verify_chain_host_workspace")
+    return n.value
+
+
+def polyspec_verify_chain_host(models, k, draft_tokens, uniforms, temperature, workspace, out=None,
+                               host_status=None, stream=None):
+    """The chain for HOST buffers (CPU tensors, ideally pinned); `workspace` is a device tensor of at least
+    polyspec_verify_chain_host_workspace bytes.  Outputs are CPU tensors, valid after the stream synchronises."""
+    lib = load_library()
+    n = len(models)
+    L = n - 1
+    B, _, V = models[0].shape
+    dt = _dt(models[0])
+    rows = [int(m.shape[1]) for m in models]
+    kmax = max(int(x) for x in k)
+    for t in list(models) + [draft_tokens, uniforms]:
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("polyspec_verify_chain_host takes contiguous CPU tensors")
+    if not workspace.is_cuda:
+        raise ValueError("the workspace must be a CUDA tensor")
+    if out is None:
+        out = chain_outputs(L, B, kmax, "cpu", pin=True)
+    if host_status is None:
+        host_status = torch.zeros(1, dtype=torch.int32, pin_memory=True)
+    arr = (ModelLogits * n)(*[ModelLogits(m.data_ptr(), r) for m, r in zip(models, rows)])
+    with torch.cuda.device(workspace.device):
+        st = lib.polyspec_verify_chain_host(arr, n, _int_array(k), _ptr(draft_tokens), _ptr(uniforms), B, V, dt,
+                                            float(temperature), _ptr(out["accepted_len"]), _ptr(out["block_len"]),
+                                            _ptr(out["out_tokens"]), _ptr(out["out_len"]), _ptr(host_status),
+                                            _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "polyspec_verify_chain_host")
+    out["host_status"] = host_status
+    return out
+
+
+# ------------------------------------------------------------------ verify_from_hidden
+def polyspec_verify_from_hidden_workspace(B: int, k: int, V: int, d_p: int, d_q: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().polyspec_verify_from_hidden_workspace(B, k, V, d_p, d_q, ctypes.byref(n)),
+           "polyspec_verify_from_hidden_workspace")
+    return n.value
+
+
+def polyspec_verify_from_hidden(hidden_p, W_p, hidden_q, W_q, draft_tokens, uniforms, temperature, block_len=None,
+                                want_probs=False, workspace=None, out=None, device_status=None, stream=None):
+    """verify_level with the LM-head projection fused in front: hidden_p [B,k+1,d_p], W_p [V,d_p],
+    hidden_q [B,rows_q>=k,d_q], W_q [V,d_q], all bf16."""
+    lib = load_library()
+    _dev_check(hidden_p, W_p, hidden_q, W_q, draft_tokens, uniforms, block_len)
+    B, rows_p, d_p = hidden_p.shape
+    _, rows_q, d_q = hidden_q.shape
+    V = W_p.shape[0]
+    k = draft_tokens.shape[1]
+    if rows_p != k + 1 or W_q.shape[0] != V or W_p.shape[1] != d_p or W_q.shape[1] != d_q or hidden_q.shape[0] != B:
+        raise ValueError("shapes must be hidden_p [B,k+1,d_p], W_p [V,d_p], hidden_q [B,rows_q,d_q], W_q [V,d_q]")
+    if any(t.dtype != torch.bfloat16 for t in (hidden_p, W_p, hidden_q, W_q)):
+        raise TypeError("hidden states and LM-head weights must be bfloat16")
+    dev = hidden_p.device
+    if workspace is None:
+        workspace = _workspace(polyspec_verify_from_hidden_workspace(B, k, V, d_p, d_q), dev)
+    if out is None:
+        out = {"accepted_len": torch.empty(B, dtype=torch.int32, device=dev),
+               "next_token": torch.empty(B, dtype=torch.int32, device=dev)}
+        if want_probs:
+            out["p_at_draft"] = torch.empty((B, k), dtype=torch.float32, device=dev)
+            out["q_at_draft"] = torch.empty((B, k), dtype=torch.float32, device=dev)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib.polyspec_verify_from_hidden(
+        _ptr(hidden_p), _ptr(W_p), _ptr(hidden_q), _ptr(W_q), rows_q, _ptr(draft_tokens), _ptr(uniforms), _ptr(block_len),
+        B, k, V, d_p, d_q, float(temperature), _ptr(out["accepted_len"]), _ptr(out["next_token"]),
+        _ptr(out.get("p_at_draft")), _ptr(out.get("q_at_draft")), _ptr(device_status),
+        _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "polyspec_verify_from_hidden")
+    out["device_status"] = device_status
+    return out

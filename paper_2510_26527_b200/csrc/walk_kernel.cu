@@ -1,0 +1,370 @@
+// Decision and sampling: one CTA walks one sequence up the chain, level by level
+// (Section 3.1: the drafted block is "verified in ascending order by M_{n-1}, ..., M_1").
+// Per level (Algorithm 1: Verify with a break at the first failure, then the token that
+// replaces the first rejected one, or the bonus token after a fully accepted block):
+//   1. merge the row-statistics partials of the rows this level needs;
+//   2. gather P_j(x_j), Q_j(x_j), test u_j * Q <= P in double precision, ballot for the
+//      first rejection -> accepted length a;
+//   3. one pass over row a of p (and of q unless this is the bonus row): residual
+//      max(0, P - Q) per element, per-tile sums, a scan of the tile sums, then a rescan of
+//      the one tile that contains u_s * total -> next token (inverse CDF, ascending order);
+//   4. the emitted stream (x_1..x_a, next) becomes the block of the level above.
+// Levels of one sequence depend on each other; sequences do not, so there is no
+// inter-CTA communication and no waiting of any kind.
+#include "polyspec_kernels.cuh"
+
+namespace polyspec {
+namespace {
+
+constexpr int kWalkThreads = 512;
+constexpr int kWalkWarps = kWalkThreads / 32;
+
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ uint4 ld_nc(const void* p)
+{
+    uint4 r;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+template <int DT> __device__ __forceinline__ float load_logit(const void* row, int v)
+{
+    if (DT == POLYSPEC_BF16)
+        return __uint_as_float(static_cast<uint32_t>(static_cast<const unsigned short*>(row)[v]) << 16);
+    return static_cast<const float*>(row)[v];
+}
+
+// Eight consecutive logits starting at element v (v a multiple of 8, inside the row).
+template <int DT> __device__ __forceinline__ void load8(const void* row, int v, float* z)
+{
+    if (DT == POLYSPEC_BF16) {
+        const uint4 r = ld_nc(static_cast<const unsigned short*>(row) + v);
+        z[0] = __uint_as_float(r.x << 16); z[1] = __uint_as_float(r.x & 0xffff0000u);
+        z[2] = __uint_as_float(r.y << 16); z[3] = __uint_as_float(r.y & 0xffff0000u);
+        z[4] = __uint_as_float(r.z << 16); z[5] = __uint_as_float(r.z & 0xffff0000u);
+        z[6] = __uint_as_float(r.w << 16); z[7] = __uint_as_float(r.w & 0xffff0000u);
+    } else {
+        const uint4 a = ld_nc(static_cast<const float*>(row) + v);
+        const uint4 b = ld_nc(static_cast<const float*>(row) + v + 4);
+        z[0] = __uint_as_float(a.x); z[1] = __uint_as_float(a.y); z[2] = __uint_as_float(a.z); z[3] = __uint_as_float(a.w);
+        z[4] = __uint_as_float(b.x); z[5] = __uint_as_float(b.y); z[6] = __uint_as_float(b.z); z[7] = __uint_as_float(b.w);
+    }
+}
+
+struct RowStat {      // sum_v 2^(z_v * c - E) = Z
+    float E;
+    double Z;
+};
+
+__device__ __forceinline__ RowStat merge_partials(const float2* part, int parts)
+{
+    float E = kEmptyRef;
+    for (int i = 0; i < parts; ++i) E = fmaxf(E, part[i].x);
+    double Z = 0.0;
+    for (int i = 0; i < parts; ++i) {
+        const float2 ps = part[i];
+        const float d = ps.x - E;                       // integer-valued, <= 0
+        Z += (d < -1000.0f) ? static_cast<double>(ps.y) * 0.0 : ldexp(static_cast<double>(ps.y), static_cast<int>(d));
+    }
+    RowStat r;
+    r.E = E;
+    r.Z = Z;
+    return r;
+}
+
+__device__ __forceinline__ bool stat_ok(const RowStat& s) { return s.Z > 0.0 && s.Z < 1.0e300; }   // false for NaN too
+
+// The residual (or, without q, the probability) of one element, in a fixed operation order
+// so that the sum pass and the rescan produce identical values.
+__device__ __forceinline__ float resid(float zp, float zq, float c, float Ep, float iZp, float Eq, float iZq, bool use_q)
+{
+    const float pv = __fmul_rn(ex2f(__fmaf_rn(zp, c, -Ep)), iZp);
+    if (!use_q) return pv;
+    const float qv = __fmul_rn(ex2f(__fmaf_rn(zq, c, -Eq)), iZq);
+    return fmaxf(0.0f, __fsub_rn(pv, qv));
+}
+
+__device__ __forceinline__ float sum8(const float* r)
+{
+    return __fadd_rn(__fadd_rn(__fadd_rn(r[0], r[1]), __fadd_rn(r[2], r[3])),
+                     __fadd_rn(__fadd_rn(r[4], r[5]), __fadd_rn(r[6], r[7])));
+}
+
+template <int DT>
+__device__ __forceinline__ void tile_resid(const void* prow, const void* qrow, int v, int V, float c,
+                                           float Ep, float iZp, float Eq, float iZq, bool use_q, float* r)
+{
+    if (v < V) {
+        float zp[8], zq[8];
+        load8<DT>(prow, v, zp);
+        if (use_q) load8<DT>(qrow, v, zq);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = resid(zp[e], use_q ? zq[e] : 0.0f, c, Ep, iZp, Eq, iZq, use_q);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) r[e] = 0.0f;
+    }
+}
+
+__device__ __forceinline__ double warp_incl_scan(double x, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+    }
+    return x;
+}
+
+struct SampleShared {
+    double total;
+    double prefix;     // mass before the chosen tile
+    int tile;
+    int token;
+};
+
+// Inverse CDF of the residual (use_q) or of P (bonus / fallback) at uniform u.
+// Returns the token (same value in every thread) and the total mass through *total_out.
+template <int DT>
+__device__ int sample_row(const void* prow, const void* qrow, int V, float c, RowStat sp, RowStat sq, bool use_q,
+                          float u, float* tile_sum, SampleShared* sh, double* total_out)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int ntiles = (V + kTile - 1) / kTile;
+    const float iZp = static_cast<float>(1.0 / sp.Z);
+    const float iZq = use_q ? static_cast<float>(1.0 / sq.Z) : 0.0f;
+    const float Ep = sp.E, Eq = sq.E;
+
+    for (int t = warp; t < ntiles; t += kWalkWarps) {
+        float r[8];
+        tile_resid<DT>(prow, qrow, t * kTile + lane * 8, V, c, Ep, iZp, Eq, iZq, use_q, r);
+        float x = sum8(r);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
+        if (lane == 0) tile_sum[t] = x;
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        // each lane owns a contiguous run of tiles; tile sums are added in double, in order
+        const int per = (ntiles + 31) / 32;
+        const int t0 = min(lane * per, ntiles), t1 = min(t0 + per, ntiles);
+        double mine = 0.0;
+        for (int t = t0; t < t1; ++t) mine += static_cast<double>(tile_sum[t]);
+        const double incl = warp_incl_scan(mine, lane);
+        const double total = __shfl_sync(0xffffffffu, incl, 31);
+        const double target = static_cast<double>(u) * total;
+        const unsigned hit = __ballot_sync(0xffffffffu, incl > target);
+        const unsigned has_mass = __ballot_sync(0xffffffffu, mine > 0.0);
+        // the first lane whose running sum passes the target; if the uniform was not below 1
+        // or rounding leaves none, the last lane that holds any mass
+        const int owner = hit ? (__ffs(hit) - 1) : (has_mass ? (31 - __clz(has_mass)) : -1);
+        int tile = -1;
+        double prefix = 0.0;
+        if (owner >= 0) {
+            if (lane == owner) {
+                double run = incl - mine;
+                for (int t = t0; t < t1; ++t) {
+                    const double nxt = run + static_cast<double>(tile_sum[t]);
+                    if (nxt > target) { tile = t; prefix = run; break; }
+                    run = nxt;
+                }
+                if (tile < 0) {                       // take the lane's last non-empty tile
+                    run = incl - mine;
+                    for (int t = t0; t < t1; ++t) {
+                        if (tile_sum[t] > 0.0f) { tile = t; prefix = run; }
+                        run += static_cast<double>(tile_sum[t]);
+                    }
+                }
+            }
+            tile = __shfl_sync(0xffffffffu, tile, owner);
+            prefix = __shfl_sync(0xffffffffu, prefix, owner);
+        }
+        int token = -1;
+        if (tile >= 0) {
+            float r[8];
+            tile_resid<DT>(prow, qrow, tile * kTile + lane * 8, V, c, Ep, iZp, Eq, iZq, use_q, r);
+            double lane_sum = 0.0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) lane_sum += static_cast<double>(r[e]);
+            const double lincl = warp_incl_scan(lane_sum, lane);
+            const double tt = target - prefix;
+            const unsigned lhit = __ballot_sync(0xffffffffu, lincl > tt);
+            const unsigned lpos = __ballot_sync(0xffffffffu, lane_sum > 0.0);
+            // the first lane whose running sum passes the target; if rounding leaves none, the last lane with mass
+            const int pick = lhit ? (__ffs(lhit) - 1) : (lpos ? (31 - __clz(lpos)) : -1);
+            if (pick >= 0 && lane == pick) {
+                double run = lincl - lane_sum;
+                int last_pos = -1;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    if (token < 0) {
+                        run += static_cast<double>(r[e]);
+                        if (r[e] > 0.0f) last_pos = e;
+                        if (run > tt) token = tile * kTile + lane * 8 + e;
+                    }
+                }
+                if (token < 0 && last_pos >= 0) token = tile * kTile + lane * 8 + last_pos;
+            }
+            if (pick >= 0) token = __shfl_sync(0xffffffffu, token, pick);
+        }
+        if (lane == 0) {
+            sh->total = total;
+            sh->token = token;
+        }
+    }
+    __syncthreads();
+    *total_out = sh->total;
+    const int token = sh->token;
+    __syncthreads();          // sh and tile_sum are reused by the next pass
+    return token;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kWalkThreads) walk_kernel(const WalkParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* tile_sum = reinterpret_cast<float*>(smem_raw);
+
+    __shared__ int tok[kMaxK + 2];
+    __shared__ RowStat st_p[kMaxK + 1];
+    __shared__ RowStat st_q[kMaxK + 1];
+    __shared__ int sh_a, sh_bad;
+    __shared__ SampleShared sh_sample;
+
+    constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int L = p.n_levels;
+    const size_t row_bytes = static_cast<size_t>(p.V) * ELEM;
+    const double cd = static_cast<double>(p.c);
+
+    int stream_len = p.k[L - 1];
+    if (p.bottom_len) stream_len = max(0, min(stream_len, p.bottom_len[b]));
+    if (tid < p.k[L - 1]) tok[tid] = p.draft_tokens[static_cast<size_t>(b) * p.k[L - 1] + tid];
+    __syncthreads();
+
+    bool dead = false;
+    for (int l = L - 1; l >= 0; --l) {
+        const int kl = p.k[l];
+        const size_t lb = static_cast<size_t>(l) * p.B + b;
+        if (dead) {               // an unusable input below: this level reports -1 as well
+            if (tid == 0) {
+                p.accepted_len[lb] = -1;
+                if (p.block_len) p.block_len[lb] = -1;
+                if (p.out_len) p.out_len[lb] = -1;
+            }
+            if (p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
+            continue;
+        }
+        const int m = min(kl, stream_len);
+        const int grow_p = p.t.row_begin[l] + b * p.t.rows[l];
+        const int grow_q = p.t.row_begin[l + 1] + b * p.t.rows[l + 1];
+        const char* base_p = static_cast<const char*>(p.t.logits[l]) + static_cast<size_t>(b) * p.t.rows[l] * row_bytes;
+        const char* base_q = static_cast<const char*>(p.t.logits[l + 1]) + static_cast<size_t>(b) * p.t.rows[l + 1] * row_bytes;
+
+        // 1. normalisers of p rows 0..m and q rows 0..m-1
+        if (tid <= m) st_p[tid] = merge_partials(p.partials + static_cast<size_t>(grow_p + tid) * p.parts, p.parts);
+        if (tid >= 64 && tid - 64 < m) st_q[tid - 64] = merge_partials(p.partials + static_cast<size_t>(grow_q + tid - 64) * p.parts, p.parts);
+        __syncthreads();
+
+        // 2. accept tests (warp 0; m <= 32)
+        if (tid < 32) {
+            bool rej = false, bad = false;
+            float pf = 0.0f, qf = 0.0f;
+            if (tid < m) {
+                const int x = tok[tid];
+                const RowStat sp = st_p[tid], sq = st_q[tid];
+                if (x < 0 || x >= p.V || !stat_ok(sp) || !stat_ok(sq)) {
+                    bad = true;
+                } else {
+                    const float zp = load_logit<DT>(base_p + tid * row_bytes, x);
+                    const float zq = load_logit<DT>(base_q + tid * row_bytes, x);
+                    const double P = exp2(static_cast<double>(zp) * cd - static_cast<double>(sp.E)) / sp.Z;
+                    const double Q = exp2(static_cast<double>(zq) * cd - static_cast<double>(sq.E)) / sq.Z;
+                    const double u = static_cast<double>(p.uniforms[lb * (p.kmax + 1) + tid]);
+                    rej = !(u * Q <= P);
+                    pf = static_cast<float>(P);
+                    qf = static_cast<float>(Q);
+                }
+            }
+            if (l == 0 && p.p_at && tid < kl) p.p_at[static_cast<size_t>(b) * kl + tid] = pf;
+            if (l == 0 && p.q_at && tid < kl) p.q_at[static_cast<size_t>(b) * kl + tid] = qf;
+            const unsigned rej_mask = __ballot_sync(0xffffffffu, rej);
+            const unsigned bad_mask = __ballot_sync(0xffffffffu, bad);
+            const int first_rej = rej_mask ? (__ffs(rej_mask) - 1) : m;
+            const int first_bad = bad_mask ? (__ffs(bad_mask) - 1) : m + 1;
+            if (tid == 0) {
+                int isbad = first_bad < first_rej;
+                if (!isbad && first_rej == m && !stat_ok(st_p[m])) isbad = 1;     // bonus row unusable
+                sh_a = first_rej;
+                sh_bad = isbad;
+            }
+        }
+        __syncthreads();
+        const int a = sh_a;
+        if (sh_bad) {
+            dead = true;
+            if (tid == 0) {
+                p.accepted_len[lb] = -1;
+                if (p.block_len) p.block_len[lb] = -1;
+                if (p.out_len) p.out_len[lb] = -1;
+                if (p.next_token) p.next_token[b] = -1;
+                if (p.device_status) atomicCAS(p.device_status, 0, static_cast<int>(POLYSPEC_ERR_BAD_INPUT_ON_DEVICE));
+            }
+            if (p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
+            __syncthreads();
+            continue;
+        }
+
+        // 3. replacement (a < m) or bonus (a == m) token
+        const float u_s = p.uniforms[lb * (p.kmax + 1) + p.kmax];
+        const void* prow = base_p + a * row_bytes;
+        const void* qrow = base_q + a * row_bytes;
+        bool use_q = a < m;
+        const RowStat sp = st_p[a];
+        const RowStat sq = use_q ? st_q[a] : sp;
+        double total = 0.0;
+        int next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, use_q, u_s, tile_sum, &sh_sample, &total);
+        if (use_q && !(total > 0.0)) {          // residual vanished in floating point: sample P instead
+            next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, false, u_s, tile_sum, &sh_sample, &total);
+        }
+
+        // 4. outputs and hand-off
+        if (tid == 0) {
+            p.accepted_len[lb] = a;
+            if (p.block_len) p.block_len[lb] = m;
+            if (p.out_len) p.out_len[lb] = a + 1;
+            if (p.next_token) p.next_token[b] = next;
+        }
+        if (p.out_tokens && tid <= p.kmax)
+            p.out_tokens[lb * (p.kmax + 1) + tid] = (tid < a) ? tok[tid] : (tid == a ? next : -1);
+        __syncthreads();
+        if (tid == 0) tok[a] = next;
+        stream_len = a + 1;
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p, cudaStream_t stream)
+{
+    if (p.B <= 0) return cudaSuccess;
+    const int ntiles = (p.V + kTile - 1) / kTile;
+    const size_t smem = static_cast<size_t>(ntiles) * sizeof(float);
+    if (dt == POLYSPEC_BF16)
+        walk_kernel<POLYSPEC_BF16><<<p.B, kWalkThreads, smem, stream>>>(p);
+    else
+        walk_kernel<POLYSPEC_F32><<<p.B, kWalkThreads, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace polyspec

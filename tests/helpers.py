@@ -130,3 +130,46 @@ def compare_level(gpu_a, gpu_next, ora_a, ora_next, accept_margin, sample_info, 
     if margin <= band and gpu_next in (int(prev), int(succ)) and gpu_next >= 0:
         return "tie_sample"
     return "mismatch"
+
+
+def compare_chain(gpu, ora, seqs=None, band=TIE_BAND):
+    """Compare chain outputs (dicts of numpy arrays [L, B, ...]) sequence by sequence, bottom level first.
+
+    After a counted tie the two sides walk different streams, so the levels above it are skipped
+    (counted as "skipped_after_tie").  Returns a dict of counts and a list of mismatch descriptions.
+    """
+    L, B = ora["accepted_len"].shape
+    counts = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "skipped_after_tie": 0}
+    bad = []
+    for b in (range(B) if seqs is None else seqs):
+        for l in range(L - 1, -1, -1):
+            kind = compare_level(int(gpu["accepted_len"][l, b]), int(gpu["out_tokens"][l, b, max(int(gpu["accepted_len"][l, b]), 0)]),
+                                 int(ora["accepted_len"][l, b]), int(ora["out_tokens"][l, b, max(int(ora["accepted_len"][l, b]), 0)]),
+                                 ora["accept_margin"][l, b], ora["sample_info"][l, b], band)
+            if kind == "exact":
+                same = (gpu["block_len"][l, b] == ora["block_len"][l, b] and gpu["out_len"][l, b] == ora["out_len"][l, b]
+                        and (gpu["out_tokens"][l, b] == ora["out_tokens"][l, b]).all())
+                if not same:
+                    kind = "mismatch"
+            counts[kind] += 1
+            if kind == "mismatch":
+                bad.append((b, l, int(gpu["accepted_len"][l, b]), int(ora["accepted_len"][l, b]),
+                            gpu["out_tokens"][l, b].tolist(), ora["out_tokens"][l, b].tolist()))
+                break
+            if kind != "exact":
+                counts["skipped_after_tie"] += l
+                break
+    return counts, bad
+
+
+def compare_level_batch(gpu_a, gpu_next, ora, seqs=None, band=TIE_BAND):
+    counts = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0}
+    bad = []
+    B = len(ora["accepted_len"])
+    for b in (range(B) if seqs is None else seqs):
+        kind = compare_level(int(gpu_a[b]), int(gpu_next[b]), int(ora["accepted_len"][b]), int(ora["next_token"][b]),
+                             ora["accept_margin"][b], ora["sample_info"][b], band)
+        counts[kind] += 1
+        if kind == "mismatch":
+            bad.append((b, int(gpu_a[b]), int(gpu_next[b]), int(ora["accepted_len"][b]), int(ora["next_token"][b])))
+    return counts, bad

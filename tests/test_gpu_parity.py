@@ -1,0 +1,247 @@
+"""GPU-vs-oracle parity of the logits path, through the C ABI, on the same seeded inputs.
+
+Bar: accepted lengths, block lengths, stream lengths and every emitted token bit-exact, except where
+a uniform lies within 1e-6 of its decision threshold (accept tests: |u - min(1, P/Q)|; sampling:
+distance to the chosen token's CDF edge in normalised units, and the GPU token must then be the
+neighbouring positive-mass token).  Such ties are counted, printed and bounded.  Softmax
+probabilities at the drafted tokens agree to 1e-5 relative (fp32 logits) / 2e-3 (bf16 logits).
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_26527_b200 import binding, buildlib, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    buildlib.build()
+    binding.load_library()
+    assert torch.cuda.is_available()
+
+
+def _np(out):
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def _cpu(models):
+    return [m.cpu() for m in models]
+
+
+def _run_chain(data):
+    return _np(binding.polyspec_verify_chain(data["models"], data["k"], data["draft_tokens"], data["uniforms"], data["temperature"]))
+
+
+def _oracle_chain(oracle, data, seqs=None, threads=8):
+    return oracle.verify_chain(_cpu(data["models"]), data["k"], data["draft_tokens"].cpu(), data["uniforms"].cpu(),
+                               data["temperature"], threads=threads, seqs=seqs)
+
+
+def _assert_parity(counts, bad, n_decisions, what):
+    ties = counts["tie_accept"] + counts["tie_sample"]
+    print(f"[parity] {what}: {counts}")
+    assert not bad, f"{what}: mismatches outside the 1e-6 band: {bad[:5]}"
+    assert ties <= max(2, n_decisions // 2000), f"{what}: implausibly many ties {counts}"
+
+
+# ------------------------------------------------------------------ single level, tiny shapes, every branch
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("V,k", [(8, 1), (64, 3), (1000, 2), (2048, 4), (4104, 5)])
+def test_level_tiny_shapes_every_branch(oracle, dtype, V, k):
+    B = 512
+    spec = synth.ChainSpec("tiny", 2, B, V, dtype, (k,), 0.9, 2.0, (1.2,), False)
+    d = synth.make_chain(spec, seed=V + k, device=DEV)
+    lp, lq = d["models"]
+    out = _np(binding.polyspec_verify_level(lp, lq, d["draft_tokens"], d["uniforms"][0], 0.9, want_probs=True))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), d["draft_tokens"].cpu(), d["uniforms"][0].cpu(), 0.9, threads=8)
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B * (k + 1), f"level V={V} k={k} {dtype}")
+    assert out["device_status"][0] == 0
+    assert set(np.unique(ora["accepted_len"])) == set(range(k + 1))        # every accepted length occurs
+    # probabilities at the drafted tokens (the oracle fills positions up to the first rejection)
+    tol = 1e-5 if dtype == torch.float32 else 2e-3
+    m = np.isfinite(ora["p_at"])
+    np.testing.assert_allclose(out["p_at_draft"][m], ora["p_at"][m], rtol=tol, atol=1e-30)
+    np.testing.assert_allclose(out["q_at_draft"][m], ora["q_at"][m], rtol=tol, atol=1e-30)
+
+
+def test_level_block_len_zero_to_k_and_identical_models(oracle):
+    B, k, V = 66, 5, 512
+    g = torch.Generator(device=DEV).manual_seed(1)
+    lp = torch.randn((B, k + 1, V), generator=g, device=DEV) * 3
+    lq = lp[:, :k].clone()
+    tok = torch.randint(0, V, (B, k), generator=g, device=DEV, dtype=torch.int32)
+    u = torch.from_numpy(synth.philox_uniforms(1, 1, B, k + 1)[0]).to(DEV)
+    bl = (torch.arange(B, device=DEV, dtype=torch.int32) % (k + 1)).contiguous()
+    out = _np(binding.polyspec_verify_level(lp, lq, tok, u, 1.0, block_len=bl, want_probs=True))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), 1.0, block_len=bl.cpu())
+    assert (out["accepted_len"] == bl.cpu().numpy()).all()          # p == q accepts everything presented
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B * k, "block_len 0..k, p == q")
+    # positions beyond block_len report probability 0
+    for b in range(B):
+        assert (out["p_at_draft"][b, bl[b]:] == 0).all()
+
+
+def test_level_disjoint_supports_and_masked_vocab(oracle):
+    B, k, V = 64, 3, 4096
+    g = torch.Generator(device=DEV).manual_seed(2)
+    lp = torch.randn((B, k + 1, V), generator=g, device=DEV) * 2
+    lq = torch.randn((B, k, V), generator=g, device=DEV) * 2
+    lp[:, :, : V // 2] = float("-inf")
+    lq[:, :, V // 2:] = float("-inf")
+    tok = torch.randint(0, V // 2, (B, k), generator=g, device=DEV, dtype=torch.int32)
+    u = torch.from_numpy(synth.philox_uniforms(2, 1, B, k + 1)[0]).to(DEV)
+    out = _np(binding.polyspec_verify_level(lp, lq, tok, u, 1.0))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), 1.0)
+    assert (out["accepted_len"] == 0).all() and (out["next_token"] >= V // 2).all()
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B, "disjoint supports")
+
+
+def test_level_unusable_inputs_set_status_and_minus_one(oracle):
+    B, k, V = 8, 3, 1024
+    g = torch.Generator(device=DEV).manual_seed(3)
+    lp = torch.randn((B, k + 1, V), generator=g, device=DEV)
+    lq = lp[:, :k].clone() + 0.5 * torch.randn((B, k, V), generator=g, device=DEV)
+    tok = torch.randint(0, V, (B, k), generator=g, device=DEV, dtype=torch.int32)
+    u = torch.full((B, k + 1), 1e-6, device=DEV)          # tiny uniforms: everything is accepted
+    tok[1, 0] = V                                          # token out of range at the first position
+    tok[2, 2] = -1
+    lp[3, 1, 17] = float("nan")
+    lq[4, 0] = float("-inf")                               # a row with no finite logit
+    lp[5, k, 5] = float("inf")                             # unusable bonus row
+    out = _np(binding.polyspec_verify_level(lp, lq, tok, u, 1.0))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), 1.0)
+    assert out["device_status"][0] == binding.ERR_BAD_INPUT_ON_DEVICE
+    for b in range(B):
+        if ora["status"][b] != 0:
+            assert out["accepted_len"][b] == -1 and out["next_token"][b] == -1, b
+        else:
+            assert out["accepted_len"][b] == ora["accepted_len"][b] and out["next_token"][b] == ora["next_token"][b], b
+    assert sorted(np.nonzero(ora["status"])[0].tolist()) == [1, 2, 3, 4, 5]
+
+
+def test_outputs_are_deterministic():
+    spec = synth.scaled(synth.config("cfg3"), B=8, V=20000)
+    d = synth.make_chain(spec, seed=5, device=DEV)
+    a = _run_chain(d)
+    b = _run_chain(d)
+    for key in ("accepted_len", "block_len", "out_tokens", "out_len"):
+        assert (a[key] == b[key]).all()
+
+
+# ------------------------------------------------------------------ chains, reduced sizes
+@pytest.mark.parametrize("name,B,V,sigma", [("cfg2", 24, 4096, None), ("cfg3", 16, 10000, None),
+                                            ("cfg5", 12, 8200, 0.5), ("cfg5", 12, 24, 2.0)])
+def test_chain_reduced_sizes(oracle, name, B, V, sigma):
+    spec = synth.scaled(synth.config(name, sigma=sigma), B=B, V=V)
+    d = synth.make_chain(spec, seed=7, device=DEV)
+    out = _run_chain(d)
+    ora = _oracle_chain(oracle, d)
+    counts, bad = H.compare_chain(out, ora)
+    _assert_parity(counts, bad, B * sum(spec.k), f"{name} reduced B={B} V={V}")
+    assert out["device_status"][0] == 0
+
+
+# ------------------------------------------------------------------ the benchmark configurations at full size
+def test_config1_full(oracle):
+    spec = synth.config("cfg1")
+    for seed in range(8):
+        d = synth.make_chain(spec, seed=seed, device=DEV)
+        lp, lq = d["models"]
+        out = _np(binding.polyspec_verify_level(lp, lq, d["draft_tokens"], d["uniforms"][0], 1.0, want_probs=True))
+        ora = oracle.verify_level(lp.cpu(), lq.cpu(), d["draft_tokens"].cpu(), d["uniforms"][0].cpu(), 1.0)
+        counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+        assert not bad and counts["exact"] == 1, (seed, counts, bad)
+        m = np.isfinite(ora["p_at"])
+        np.testing.assert_allclose(out["p_at_draft"][m], ora["p_at"][m], rtol=1e-5)
+        np.testing.assert_allclose(out["q_at_draft"][m], ora["q_at"][m], rtol=1e-5)
+
+
+def test_config2_full(oracle):
+    spec = synth.config("cfg2")
+    total = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "skipped_after_tie": 0}
+    for seed in range(8):
+        d = synth.make_chain(spec, seed=seed, device=DEV)
+        counts, bad = H.compare_chain(_run_chain(d), _oracle_chain(oracle, d))
+        assert not bad, (seed, bad)
+        for key in total:
+            total[key] += counts[key]
+    _assert_parity(total, [], 8 * 17, "cfg2 full, 8 seeds")
+
+
+def test_config3_full(oracle):
+    spec = synth.config("cfg3")
+    d = synth.make_chain(spec, seed=0, device=DEV)
+    out = _run_chain(d)
+    ora = _oracle_chain(oracle, d)
+    counts, bad = H.compare_chain(out, ora)
+    _assert_parity(counts, bad, 64 * 12, "cfg3 full")
+    # bf16 softmax probabilities at the bottom level, via the single-level call on the same rows
+    lv = _np(binding.polyspec_verify_level(d["models"][1].contiguous(), d["models"][2], d["draft_tokens"],
+                                           d["uniforms"][1, :, :].contiguous(), spec.temperature, want_probs=True))
+    for b in (0, 17, 63):
+        for j in (0, 5):
+            x = int(d["draft_tokens"][b, j])
+            P = oracle.softmax_row(d["models"][1][b, j].cpu(), spec.temperature)[x]
+            Q = oracle.softmax_row(d["models"][2][b, j].cpu(), spec.temperature)[x]
+            assert abs(lv["p_at_draft"][b, j] - P) <= 2e-3 * P and abs(lv["q_at_draft"][b, j] - Q) <= 2e-3 * Q
+
+
+@pytest.mark.parametrize("sigma", synth.CFG5_SIGMAS)
+def test_config5_full_size_sampled_sequences(oracle, sigma):
+    """The launch configuration the benchmark times (B=256, V=152064, four models); the oracle checks a
+    sample of the sequences one by one, and the whole batch is checked against properties that hold at
+    any size: hand-off bookkeeping and the bottom level's closed-form mean acceptance length."""
+    spec = synth.config("cfg5", sigma=sigma)
+    d = synth.make_chain(spec, seed=int(sigma * 100), device=DEV)
+    out = _run_chain(d)
+    seqs = [0, 1, 2, 3, 100, 101, 254, 255]
+    sub = [m[seqs].cpu() for m in d["models"]]
+    ora = oracle.verify_chain(sub, d["k"], d["draft_tokens"][seqs].cpu(), d["uniforms"][:, seqs].cpu().contiguous(),
+                              spec.temperature, threads=8)
+    gpu_sub = {key: out[key][:, seqs] for key in ("accepted_len", "block_len", "out_tokens", "out_len")}
+    counts, bad = H.compare_chain(gpu_sub, ora)
+    _assert_parity(counts, bad, len(seqs) * 20, f"cfg5 sigma={sigma} sampled sequences")
+    # whole batch: bookkeeping
+    k = spec.k
+    assert (out["block_len"][2] == k[2]).all()
+    assert (out["block_len"][1] == np.minimum(k[1], out["out_len"][2])).all()
+    assert (out["block_len"][0] == np.minimum(k[0], out["out_len"][1])).all()
+    assert (out["out_len"] == out["accepted_len"] + 1).all()
+    assert (out["accepted_len"] <= out["block_len"]).all() and (out["accepted_len"] >= 0).all()
+    for l in range(3):
+        for b in (5, 77, 200):
+            n = out["out_len"][l, b]
+            assert (out["out_tokens"][l, b, :n] >= 0).all() and (out["out_tokens"][l, b, n:] == -1).all()
+    # whole batch: E[a] at the bottom level = sum_j prod alpha_i, alpha from a float64 softmax on the device
+    P = torch.softmax(d["models"][2][:, :k[2]].double(), dim=-1)
+    Q = torch.softmax(d["models"][3].double(), dim=-1)
+    alpha = torch.minimum(P, Q).sum(-1)
+    expect = torch.cumprod(alpha, dim=1).sum(1).cpu().numpy()
+    diff = out["accepted_len"][2] - expect
+    se = diff.std(ddof=1) / np.sqrt(len(diff))
+    assert abs(diff.mean()) < 3 * se + 1e-9, (sigma, diff.mean(), se)
+
+
+def test_chain_host_entry_point_matches_device_entry_point():
+    spec = synth.scaled(synth.config("cfg5", sigma=1.0), B=16, V=16384)
+    d = synth.make_chain(spec, seed=9, device=DEV)
+    ref = _run_chain(d)
+    models = [m.cpu().pin_memory() for m in d["models"]]
+    rows = [m.shape[1] for m in models]
+    ws = torch.empty(binding.polyspec_verify_chain_host_workspace(d["k"], rows, spec.B, spec.V, binding.BF16),
+                     dtype=torch.uint8, device=DEV)
+    out = binding.polyspec_verify_chain_host(models, d["k"], d["draft_tokens"].cpu().pin_memory(),
+                                             d["uniforms"].cpu().pin_memory(), spec.temperature, ws)
+    torch.cuda.synchronize()
+    for key in ("accepted_len", "block_len", "out_tokens", "out_len"):
+        assert (out[key].numpy() == ref[key]).all()
+    assert out["host_status"][0] == 0
