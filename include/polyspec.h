@@ -60,7 +60,8 @@ typedef enum {
     POLYSPEC_ERR_WORKSPACE = 3,
     POLYSPEC_ERR_CUDA = 4,
     POLYSPEC_ERR_TIMEOUT = 5,
-    POLYSPEC_ERR_BAD_INPUT_ON_DEVICE = 6
+    POLYSPEC_ERR_BAD_INPUT_ON_DEVICE = 6,
+    POLYSPEC_ERR_SCRATCH_LIMIT = 7      /* problem too large for the built-in scratch of a *_static call */
 } polyspec_status;
 
 typedef enum { POLYSPEC_F32 = 0, POLYSPEC_BF16 = 1 } polyspec_dtype;
@@ -174,6 +175,37 @@ polyspec_status polyspec_verify_from_hidden(
     int B, int k, int V, int d_p, int d_q, float temperature,
     int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * polyspec_verify_level_static -- polyspec_verify_level without a workspace argument.
+ * (The paper has no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Some callers cannot give the library a workspace because they cannot allocate device
+ * memory at the point where they verify: a plugin invoked from inside a serving engine
+ * that owns every byte of the device, code running under a fixed post-start-up memory
+ * budget, a callback in which cudaMalloc is forbidden.  For them the row-statistics
+ * partials live in a fixed array of POLYSPEC_STATIC_SCRATCH_BYTES inside the library image
+ * (each GPU that loads the library holds that much until the process exits).  The call
+ * allocates nothing, neither through CUDA nor through any library.
+ *
+ *   - Inputs and outputs are the caller's, exactly as in polyspec_verify_level.
+ *   - Limit: the call needs polyspec_verify_level_workspace(B, k, V, dt) bytes; if that
+ *     exceeds POLYSPEC_STATIC_SCRATCH_BYTES it returns POLYSPEC_ERR_SCRATCH_LIMIT and launches
+ *     nothing.  (1 MiB covers e.g. B = 256, k = 8, V = 152064 in bf16.)
+ *   - The device that owns `cuda_stream` must be current.  The first call on each device
+ *     looks up the device address of the array (a one-time set-up step); make that first
+ *     call before starting any stream capture.
+ *   - All calls on a device share the one array.  A call overwrites every entry it later
+ *     reads, so leftovers from earlier calls do not matter, but two calls whose kernels
+ *     overlap on the GPU (different streams) race: serialise them.
+ */
+#define POLYSPEC_STATIC_SCRATCH_BYTES (1u << 20)
+size_t polyspec_static_scratch_bytes(void);
+polyspec_status polyspec_verify_level_static(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
+    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libpolyspec.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_INPUT_ON_DEVICE = 1, 2, 3, 4, 5, 6
+ERR_SCRATCH_LIMIT = 7
 F32, BF16 = 0, 1
 MAX_K, MAX_MODELS = 32, 8
 
@@ -27,6 +28,7 @@ EXPORTS = (
     "polyspec_chain_row_stats", "polyspec_chain_walk",
     "polyspec_verify_chain_host_workspace", "polyspec_verify_chain_host",
     "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden",
+    "polyspec_static_scratch_bytes", "polyspec_verify_level_static",
 )
 
 
@@ -83,6 +85,11 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_from_hidden.restype = ci
     lib.polyspec_verify_from_hidden.argtypes = [vp, vp, vp, vp, ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf,
                                                 i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
+    lib.polyspec_static_scratch_bytes.restype = sz
+    lib.polyspec_static_scratch_bytes.argtypes = []
+    lib.polyspec_verify_level_static.restype = ci
+    lib.polyspec_verify_level_static.argtypes = [vp, vp, i32p, f32p, i32p, ci, ci, ci, ci, cf,
+                                                 i32p, i32p, f32p, f32p, i32p, vp]
     _lib = lib
     return lib
 
@@ -350,4 +357,30 @@ def polyspec_verify_from_hidden(hidden_p, W_p, hidden_q, W_q, draft_tokens, unif
         _ptr(workspace), workspace.numel(), _stream(stream))
     _check(st, "polyspec_verify_from_hidden")
     out["device_status"] = device_status
+    return out
+
+
+# ------------------------------------------------------------------ verify_level without a workspace
+def polyspec_static_scratch_bytes() -> int:
+    return int(load_library().polyspec_static_scratch_bytes())
+
+
+def polyspec_verify_level_static(logits_p, logits_q, draft_tokens, uniforms, temperature, out, block_len=None,
+                                 device_status=None, stream=None):
+    """polyspec_verify_level for callers that cannot allocate device memory: no workspace is passed, the
+    library's built-in scratch array is used, and this wrapper allocates nothing either -- `out` must hold
+    the caller's own accepted_len / next_token (and optionally p_at_draft / q_at_draft) device tensors.
+    Raises PolyspecError(ERR_SCRATCH_LIMIT) when the problem needs more than polyspec_static_scratch_bytes()."""
+    lib = load_library()
+    _dev_check(logits_p, logits_q, draft_tokens, uniforms, block_len)
+    B, rows_p, V = logits_p.shape
+    k = draft_tokens.shape[1]
+    if rows_p != k + 1 or tuple(logits_q.shape) != (B, k, V) or tuple(uniforms.shape) != (B, k + 1):
+        raise ValueError("shapes must be logits_p [B,k+1,V], logits_q [B,k,V], draft_tokens [B,k], uniforms [B,k+1]")
+    with torch.cuda.device(logits_p.device):
+        st = lib.polyspec_verify_level_static(
+            _ptr(logits_p), _ptr(logits_q), _ptr(draft_tokens), _ptr(uniforms), _ptr(block_len),
+            B, k, V, _dt(logits_p), float(temperature), _ptr(out["accepted_len"]), _ptr(out["next_token"]),
+            _ptr(out.get("p_at_draft")), _ptr(out.get("q_at_draft")), _ptr(device_status), _stream(stream))
+    _check(st, "polyspec_verify_level_static")
     return out

@@ -181,6 +181,7 @@ const char* polyspec_status_string(polyspec_status s)
         case POLYSPEC_ERR_CUDA: return "CUDA error";
         case POLYSPEC_ERR_TIMEOUT: return "bounded wait expired on the device";
         case POLYSPEC_ERR_BAD_INPUT_ON_DEVICE: return "unusable input found on the device (token out of range or unusable logits row)";
+        case POLYSPEC_ERR_SCRATCH_LIMIT: return "problem too large for the built-in scratch of a *_static call";
     }
     return "unknown status";
 }
