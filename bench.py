@@ -295,7 +295,7 @@ def run_gpu(args, spec):
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": workload_name(args, spec), "seed": args.seed,
                        "l2": f"inputs {logits_bytes / 1e9:.3f} GB per step, larger than the 126 MB L2; no flush needed"
-                             if logits_bytes > 4 * 126e6 else "inputs fit in L2: L2-warm timing",
+                             if logits_bytes > 2 * 126e6 else "inputs fit in L2: L2-warm timing",
                        "parallelism": f"{world} independent replicas, batch sharded, no collective"},
             "gpu_launches": 2 * args.steps,
             "emitted_tokens_per_s": emitted_all * args.steps / (elapsed_ms * 1e-3),

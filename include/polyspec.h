@@ -39,6 +39,9 @@
  *     holding NaN / +inf or no finite logit) never trap: the affected sequence gets
  *     accepted_len = next_token = -1 (and -1 in every later level of a chain) and
  *     *device_status is set to POLYSPEC_ERR_BAD_INPUT_ON_DEVICE.
+ *   - No kernel waits without a limit.  Should a wait on the copy engine ever run out,
+ *     *device_status becomes POLYSPEC_ERR_TIMEOUT, the outputs of that call are undefined,
+ *     and the kernels still return.
  */
 #ifndef POLYSPEC_H
 #define POLYSPEC_H
@@ -134,7 +137,8 @@ polyspec_status polyspec_verify_chain(
  */
 polyspec_status polyspec_chain_row_stats(
     const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */, int B, int V,
-    polyspec_dtype dt, float temperature, void* workspace, size_t workspace_bytes, void* cuda_stream);
+    polyspec_dtype dt, float temperature, int32_t* device_status, void* workspace, size_t workspace_bytes,
+    void* cuda_stream);
 polyspec_status polyspec_chain_walk(
     const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */,
     const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,

@@ -72,7 +72,7 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_chain.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, i32p, f32p, ci, ci, ci, cf,
                                           i32p, i32p, i32p, i32p, i32p, vp, sz, vp]
     lib.polyspec_chain_row_stats.restype = ci
-    lib.polyspec_chain_row_stats.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, vp, sz, vp]
+    lib.polyspec_chain_row_stats.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, i32p, vp, sz, vp]
     lib.polyspec_chain_walk.restype = ci
     lib.polyspec_chain_walk.argtypes = lib.polyspec_verify_chain.argtypes
     lib.polyspec_verify_chain_host_workspace.restype = ci
@@ -270,7 +270,7 @@ class ChainCall:
 
     def row_stats(self):
         _check(self.lib.polyspec_chain_row_stats(self._arr, self.n, self._k, self.B, self.V, self.dt, self.temperature,
-                                                 _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)),
+                                                 _ptr(self.device_status), _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)),
                "polyspec_chain_row_stats")
 
     def walk(self):

@@ -94,6 +94,7 @@ polyspec_status prepare_chain(const ChainArgs& a, StatsPlan* pl, StatsParams* sp
     sp->n_items = static_cast<int>(pl->n_items);
     sp->c = static_cast<float>(kLog2e / static_cast<double>(a.temperature));
     sp->partials = static_cast<float2*>(a.workspace);
+    sp->status = a.device_status;
     return POLYSPEC_OK;
 }
 
@@ -251,10 +252,11 @@ polyspec_status polyspec_verify_chain(
 
 polyspec_status polyspec_chain_row_stats(
     const polyspec_model_logits* models, int n_models, const int* k, int B, int V, polyspec_dtype dt,
-    float temperature, void* workspace, size_t workspace_bytes, void* cuda_stream)
+    float temperature, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
     if (!models || !k || n_models < 2 || n_models > kMaxModels) return POLYSPEC_ERR_INVALID_ARG;
-    const ChainArgs a = chain_args(models, n_models, k, B, V, dt, temperature, workspace, workspace_bytes, cuda_stream);
+    ChainArgs a = chain_args(models, n_models, k, B, V, dt, temperature, workspace, workspace_bytes, cuda_stream);
+    a.device_status = device_status;
     return run_stats(a);
 }
 

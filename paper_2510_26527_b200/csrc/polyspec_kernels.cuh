@@ -42,6 +42,7 @@ struct StatsParams {
     int n_items;
     float c;
     float2* partials;   // [total rows, parts]
+    int32_t* status;    // [1] or nullptr: receives POLYSPEC_ERR_TIMEOUT if a bounded wait expires
 };
 
 // Decision + sampling pass: one CTA walks one sequence up the chain.

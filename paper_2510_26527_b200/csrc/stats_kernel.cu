@@ -2,24 +2,69 @@
 // read exactly once (the distribution p_i(x | x_<=t) over the vocabulary of Section 3.1
 // needs it for each drafted position before Algorithm 1's Verify can run).
 //
-// HBM-bound: each element costs one FFMA, one ex2 and one add.  Every thread keeps an
-// online pair (E, s) with  sum 2^(z*c - E) = s  and E an INTEGER-valued reference at or
-// just above its running maximum of z*c, c = log2(e)/T.  Because E is an integer,
-// rebasing s when the maximum grows, and merging pairs across lanes, warps and segments,
-// are exact multiplications by powers of two: no second exponential is ever spent.
+// HBM-bound.  One persistent CTA per SM, and inside it every warp is a self-contained
+// pipeline: lane 0 streams the warp's row segments into the warp's private ring of
+// shared-memory stages with 1-D bulk TMA copies (cp.async.bulk, completion on an
+// mbarrier), a few stages ahead of the lanes that read them back with conflict-free
+// 128-bit shared loads.  Warps never synchronise with each other, so their load, ALU and
+// ex2 phases drift apart and overlap on the SM's pipes.  Each element costs one FFMA, one
+// ex2 and one add.  Every thread keeps an online pair (E, s) with  sum 2^(z*c - E) = s
+// and E an INTEGER-valued reference at or just above its running maximum of z*c,
+// c = log2(e)/T.  Because E is an integer, rebasing s when the maximum grows, and merging
+// pairs across lanes and segments, are exact multiplications by powers of two: no second
+// exponential is ever spent.
+//
+// Every wait on an mbarrier is bounded.  If one expires the warp records
+// POLYSPEC_ERR_TIMEOUT, lets the copies it has in flight land (again bounded) and returns;
+// the outputs of that launch are then meaningless.
 #include "polyspec_kernels.cuh"
 
 namespace polyspec {
 namespace {
 
-constexpr int kStatsThreads = 256;
-constexpr int kUnroll = 4;   // 16-byte vectors in flight per thread
+constexpr int kChunkBytes = 2048;                 // one bulk copy = one warp-wide sweep of 4 vectors per lane
+constexpr int kStages = 4;                        // per-warp ring depth
+constexpr int kWarps = 24;
+constexpr int kStatsThreads = kWarps * 32;
+constexpr int kVecPerLane = kChunkBytes / 16 / 32;   // 4
+constexpr uint32_t kSpinLimit = 1u << 20;         // try_wait attempts before giving up
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p)
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
 {
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
     return r;
 }
 
@@ -58,45 +103,118 @@ template <> struct Elems<POLYSPEC_F32> {
     static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
 };
 
+// Where work item `item` lives: first byte and byte count of its row segment.
 template <int DT>
-__global__ void __launch_bounds__(kStatsThreads) stats_kernel(const StatsParams p)
+__device__ __forceinline__ void item_span(const StatsParams& p, int item, const char** src, uint32_t* bytes)
+{
+    constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
+    const int grow = item / p.parts;
+    const int part = item - grow * p.parts;
+    int mi = 0;
+    while (mi + 1 < p.t.n_models && grow >= p.t.row_begin[mi + 1]) ++mi;
+    const int v0 = part * p.seg;
+    const int v1 = min(p.V, v0 + p.seg);
+    *src = static_cast<const char*>(p.t.logits[mi]) + (static_cast<size_t>(grow - p.t.row_begin[mi]) * p.V + v0) * ELEM;
+    *bytes = static_cast<uint32_t>((v1 - v0) * ELEM);
+}
+
+// A warp's position in its list of chunks: work item (row segment) and byte offset inside it.
+struct ChunkCursor {
+    int item;
+    uint32_t off, bytes;
+    const char* src;
+};
+
+template <int DT>
+__device__ __forceinline__ void cursor_open(const StatsParams& p, ChunkCursor& cur)
+{
+    if (cur.item < p.n_items) item_span<DT>(p, cur.item, &cur.src, &cur.bytes);
+    cur.off = 0;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsParams p)
 {
     using EL = Elems<DT>;
     constexpr int EPV = EL::per_vec;
-    constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
-    __shared__ float2 warp_part[2][kStatsThreads / 32];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned char* ring = smem_raw + static_cast<size_t>(warp) * kStages * kChunkBytes;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + static_cast<size_t>(kWarps) * kStages * kChunkBytes)
+                               + warp * kStages;
+    if (lane == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    // consecutive items go to different CTAs: small problems still spread over every SM
+    const int stride = gridDim.x * kWarps;
     const float c = p.c;
-    int parity = 0;
-    for (int item = blockIdx.x; item < p.n_items; item += gridDim.x, parity ^= 1) {
-        const int grow = item / p.parts;
-        const int part = item - grow * p.parts;
-        int mi = 0;
-        while (mi + 1 < p.t.n_models && grow >= p.t.row_begin[mi + 1]) ++mi;
-        const char* base = static_cast<const char*>(p.t.logits[mi]);
-        const uint4* src = reinterpret_cast<const uint4*>(base + static_cast<size_t>(grow - p.t.row_begin[mi]) * p.V * ELEM)
-                           + (static_cast<size_t>(part) * p.seg) / EPV;
-        const int v0 = part * p.seg;
-        const int v1 = min(p.V, v0 + p.seg);
-        const int nvec = (v1 - v0) / EPV;
+
+    ChunkCursor ahead;            // next chunk to request (lane 0 runs the copies kStages-1 ahead)
+    ahead.item = warp * gridDim.x + blockIdx.x;
+    cursor_open<DT>(p, ahead);
+    uint32_t issued = 0, done = 0;
+
+    auto issue_one = [&]() {
+        if (ahead.item >= p.n_items) return;
+        const uint32_t n = min(static_cast<uint32_t>(kChunkBytes), ahead.bytes - ahead.off);
+        if (lane == 0) {
+            const uint32_t stage = issued % kStages;
+            const uint32_t bar = smem_u32(&bars[stage]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic reads of this stage are done
+            mbar_arrive_expect_tx(bar, n);
+            bulk_copy_g2s(smem_u32(ring + stage * kChunkBytes), ahead.src + ahead.off, n, bar);
+        }
+        ++issued;
+        ahead.off += n;
+        if (ahead.off >= ahead.bytes) {
+            ahead.item += stride;
+            cursor_open<DT>(p, ahead);
+        }
+    };
+
+#pragma unroll 1
+    for (int s = 0; s < kStages - 1; ++s) issue_one();
+
+    for (int item = warp * gridDim.x + blockIdx.x; item < p.n_items; item += stride) {
+        const char* src;
+        uint32_t bytes;
+        item_span<DT>(p, item, &src, &bytes);
 
         float E = kEmptyRef;
-        float s[kUnroll];
+        float s[kVecPerLane];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) s[u] = 0.0f;
+        for (int u = 0; u < kVecPerLane; ++u) s[u] = 0.0f;
 
-        for (int i = threadIdx.x; i < nvec; i += kStatsThreads * kUnroll) {
-            uint4 r[kUnroll];
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const int idx = i + u * kStatsThreads;
-                r[u] = (idx < nvec) ? ld_stream(src + idx) : EL::neg_inf();
+        for (uint32_t off = 0; off < bytes; off += kChunkBytes, ++done) {
+            __syncwarp();          // every lane has finished reading the stage the next copy will overwrite
+            issue_one();
+            const uint32_t stage = done % kStages;
+            const bool ok = wait_bounded(smem_u32(&bars[stage]), (done / kStages) & 1u);
+            if (!__all_sync(0xffffffffu, ok)) {
+                if (lane == 0) {
+                    if (p.status) atomicCAS(p.status, 0, static_cast<int>(POLYSPEC_ERR_TIMEOUT));
+                    for (uint32_t j = done; j < issued; ++j)      // let the copies in flight land
+                        wait_bounded(smem_u32(&bars[j % kStages]), (j / kStages) & 1u);
+                }
+                return;
             }
-            float z[kUnroll][EPV];
+            const int nvec = static_cast<int>(min(static_cast<uint32_t>(kChunkBytes), bytes - off) >> 4);
+            const uint32_t base = smem_u32(ring + stage * kChunkBytes);
+            uint4 r[kVecPerLane];
+#pragma unroll
+            for (int u = 0; u < kVecPerLane; ++u) {
+                const int idx = lane + u * 32;
+                r[u] = (idx < nvec) ? ld_shared_v4(base + idx * 16) : EL::neg_inf();
+            }
+            float z[kVecPerLane][EPV];
             float M = -INFINITY;
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
+            for (int u = 0; u < kVecPerLane; ++u) {
                 EL::unpack(r[u], z[u]);
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) M = fmaxf(M, z[u][e]);
@@ -105,11 +223,11 @@ __global__ void __launch_bounds__(kStatsThreads) stats_kernel(const StatsParams 
             if (En > E) {
                 const float sc = pow2_neg(E - En);
 #pragma unroll
-                for (int u = 0; u < kUnroll; ++u) s[u] *= sc;
+                for (int u = 0; u < kVecPerLane; ++u) s[u] *= sc;
                 E = En;
             }
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u)
+            for (int u = 0; u < kVecPerLane; ++u)
 #pragma unroll
                 for (int e = 0; e < EPV; ++e) s[u] += ex2f(__fmaf_rn(z[u][e], c, -E));
         }
@@ -121,35 +239,25 @@ __global__ void __launch_bounds__(kStatsThreads) stats_kernel(const StatsParams 
         float sw = ((s[0] + s[1]) + (s[2] + s[3])) * pow2_neg(E - Ew);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(0xffffffffu, sw, o);
-        if (lane == 0) warp_part[parity][warp] = make_float2(Ew, sw);
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float Eb = kEmptyRef;
-#pragma unroll
-            for (int w = 0; w < kStatsThreads / 32; ++w) Eb = fmaxf(Eb, warp_part[parity][w].x);
-            float sb = 0.0f;
-#pragma unroll
-            for (int w = 0; w < kStatsThreads / 32; ++w) sb += warp_part[parity][w].y * pow2_neg(warp_part[parity][w].x - Eb);
-            p.partials[item] = make_float2(Eb, sb);
-        }
-        // warp_part[parity] is next written two items later, after the barrier of the item in between
+        if (lane == 0) p.partials[item] = make_float2(Ew, sw);
     }
 }
 
-int g_sm_count = 0;
-int g_occ[2] = {0, 0};
+constexpr int kMaxDevices = 64;
+int g_sm_count[kMaxDevices] = {0};     // per device: SM count, filled together with the kernels' shared-memory opt-in
+constexpr size_t kStatsSmemBytes = static_cast<size_t>(kWarps) * kStages * (kChunkBytes + sizeof(unsigned long long));
 
 }  // namespace
 
 StatsPlan plan_stats(long long total_rows, int V, polyspec_dtype dt)
 {
-    (void)dt;
-    // Aim for several work items per SM even when there are few rows; a segment is a
-    // multiple of 2048 elements (256 threads x one 8-element vector).
+    // A segment (one warp's work item) is a multiple of 2048 elements and at most 16 KiB; few
+    // rows are cut finer so that every SM still gets several work items per warp.
+    const long long seg_max = 16384LL / (dt == POLYSPEC_BF16 ? 2 : 4);
     const long long total = total_rows * static_cast<long long>(V);
-    long long seg = (total / (148LL * 8) + 2047) / 2048 * 2048;
+    long long seg = (total / (148LL * kWarps * 4) + 2047) / 2048 * 2048;
     if (seg < 2048) seg = 2048;
-    if (seg > 16384) seg = 16384;
+    if (seg > seg_max) seg = seg_max;
     StatsPlan pl;
     pl.seg = static_cast<int>(seg);
     pl.parts = static_cast<int>((V + seg - 1) / seg);
@@ -162,27 +270,27 @@ StatsPlan plan_stats(long long total_rows, int V, polyspec_dtype dt)
 cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t stream)
 {
     if (p.n_items <= 0) return cudaSuccess;
-    if (g_sm_count == 0) {
-        int dev = 0, sms = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (g_sm_count[dev] == 0) {
+        int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        int o0 = 0, o1 = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o0, stats_kernel<POLYSPEC_F32>, kStatsThreads, 0);
+        e = cudaFuncSetAttribute(stats_kernel<POLYSPEC_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kStatsSmemBytes));
         if (e != cudaSuccess) return e;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o1, stats_kernel<POLYSPEC_BF16>, kStatsThreads, 0);
+        e = cudaFuncSetAttribute(stats_kernel<POLYSPEC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(kStatsSmemBytes));
         if (e != cudaSuccess) return e;
-        g_occ[0] = o0 > 0 ? o0 : 1;
-        g_occ[1] = o1 > 0 ? o1 : 1;
-        g_sm_count = sms > 0 ? sms : 148;
+        g_sm_count[dev] = sms > 0 ? sms : 148;
     }
-    const int resident = g_sm_count * g_occ[dt == POLYSPEC_BF16 ? 1 : 0];
-    const int grid = p.n_items < resident ? p.n_items : resident;
+    const int grid = p.n_items < g_sm_count[dev] ? p.n_items : g_sm_count[dev];   // one CTA per SM
     if (dt == POLYSPEC_BF16)
-        stats_kernel<POLYSPEC_BF16><<<grid, kStatsThreads, 0, stream>>>(p);
+        stats_kernel<POLYSPEC_BF16><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
     else
-        stats_kernel<POLYSPEC_F32><<<grid, kStatsThreads, 0, stream>>>(p);
+        stats_kernel<POLYSPEC_F32><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
     return cudaGetLastError();
 }
 
