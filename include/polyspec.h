@@ -181,6 +181,17 @@ polyspec_status polyspec_verify_from_hidden(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * polyspec_lm_head -- the projection of polyspec_verify_from_hidden on its own (the last op
+ * of a model forward in Algorithm 1): logits[r, v] = sum_d hidden[r, d] * W[v, d].
+ *
+ *   hidden  [rows, d] bf16, W [V, d] bf16, both row-major and 16-byte aligned; d a multiple of 64
+ *   logits  out [rows, V] fp32, 16-byte aligned
+ *   No workspace.  device_status as above (only POLYSPEC_ERR_TIMEOUT can be reported here).
+ */
+polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, int V, int d, float* logits,
+                                 int32_t* device_status, void* cuda_stream);
+
+/*
  * polyspec_verify_level_static -- polyspec_verify_level without a workspace argument.
  * (The paper has no counterpart to this call; it exists for integration reasons only.)
  *

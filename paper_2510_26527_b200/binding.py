@@ -27,7 +27,7 @@ EXPORTS = (
     "polyspec_verify_chain_workspace", "polyspec_verify_chain",
     "polyspec_chain_row_stats", "polyspec_chain_walk",
     "polyspec_verify_chain_host_workspace", "polyspec_verify_chain_host",
-    "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden",
+    "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden", "polyspec_lm_head",
     "polyspec_static_scratch_bytes", "polyspec_verify_level_static",
 )
 
@@ -85,6 +85,8 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_from_hidden.restype = ci
     lib.polyspec_verify_from_hidden.argtypes = [vp, vp, vp, vp, ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf,
                                                 i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
+    lib.polyspec_lm_head.restype = ci
+    lib.polyspec_lm_head.argtypes = [vp, vp, ci, ci, ci, f32p, i32p, vp]
     lib.polyspec_static_scratch_bytes.restype = sz
     lib.polyspec_static_scratch_bytes.argtypes = []
     lib.polyspec_verify_level_static.restype = ci
@@ -358,6 +360,27 @@ def polyspec_verify_from_hidden(hidden_p, W_p, hidden_q, W_q, draft_tokens, unif
     _check(st, "polyspec_verify_from_hidden")
     out["device_status"] = device_status
     return out
+
+
+def polyspec_lm_head(hidden, W, out=None, device_status=None, stream=None):
+    """The projection alone: hidden [..., d] bf16, W [V, d] bf16 -> fp32 logits [..., V]."""
+    lib = load_library()
+    _dev_check(hidden, W, out)
+    if hidden.dtype != torch.bfloat16 or W.dtype != torch.bfloat16:
+        raise TypeError("hidden states and LM-head weights must be bfloat16")
+    d = hidden.shape[-1]
+    rows = hidden.numel() // d
+    V = W.shape[0]
+    if W.shape[1] != d:
+        raise ValueError("hidden [..., d] and W [V, d] must share d")
+    if out is None:
+        out = torch.empty(tuple(hidden.shape[:-1]) + (V,), dtype=torch.float32, device=hidden.device)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=hidden.device)
+    with torch.cuda.device(hidden.device):
+        st = lib.polyspec_lm_head(_ptr(hidden), _ptr(W), rows, V, d, _ptr(out), _ptr(device_status), _stream(stream))
+    _check(st, "polyspec_lm_head")
+    return out, device_status
 
 
 # ------------------------------------------------------------------ verify_level without a workspace

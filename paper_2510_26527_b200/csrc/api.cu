@@ -370,6 +370,17 @@ polyspec_status polyspec_verify_chain_host(
     return POLYSPEC_OK;
 }
 
+polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, int V, int d, float* logits,
+                                 int32_t* device_status, void* cuda_stream)
+{
+    if (!hidden || !W || !logits || rows <= 0 || V <= 0 || d <= 0) return POLYSPEC_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(W) || !aligned16(logits)) return POLYSPEC_ERR_INVALID_ARG;
+    if (d % 64 != 0 || static_cast<long long>(rows) * V > 0x7fffffffLL * 16) return POLYSPEC_ERR_UNSUPPORTED;
+    const LmHeadProblem pr = {hidden, W, rows, d, logits};
+    if (launch_lmhead(&pr, 1, V, device_status, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    return POLYSPEC_OK;
+}
+
 // Workspace of the fused call: fp32 logits of both models (written by the projection, read
 // back by the statistics pass and, for one row pair per sequence, by the sampling pass),
 // then the partials.
@@ -425,8 +436,8 @@ polyspec_status polyspec_verify_from_hidden(
     char* ws = static_cast<char*>(workspace);
     float* lp = reinterpret_cast<float*>(ws + f.logits_p);
     float* lq = reinterpret_cast<float*>(ws + f.logits_q);
-    if (launch_lmhead(hidden_p, W_p, B * (k + 1), V, d_p, lp, device_status, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (launch_lmhead(hidden_q, W_q, B * rows_q, V, d_q, lq, device_status, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    const LmHeadProblem probs[2] = {{hidden_p, W_p, B * (k + 1), d_p, lp}, {hidden_q, W_q, B * rows_q, d_q, lq}};
+    if (launch_lmhead(probs, 2, V, device_status, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
 
     ChainArgs a;
     std::memset(&a, 0, sizeof a);

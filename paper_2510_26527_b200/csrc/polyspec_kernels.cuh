@@ -83,10 +83,16 @@ StatsPlan plan_stats(long long total_rows, int V, polyspec_dtype dt);
 cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t stream);
 cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p, cudaStream_t stream);
 
-// LM-head projection on the tensor cores: out[r, v] = sum_d hidden[r, d] * W[v, d],
-// bf16 inputs, fp32 output [rows, V].
-size_t lmhead_workspace_bytes(int rows, int V, int d);
-cudaError_t launch_lmhead(const void* hidden, const void* W, int rows, int V, int d, float* out,
-                          int32_t* device_status, cudaStream_t stream);
+// LM-head projection on the tensor cores: out[r, v] = sum_d hidden[r, d] * W[v, d], bf16 inputs
+// (hidden [rows, d], W [V, d], both row-major and 16-byte aligned, d a multiple of 64), fp32
+// output [rows, V].  Up to two projections (the verifier's and the drafter's) share one launch.
+struct LmHeadProblem {
+    const void* hidden;
+    const void* W;
+    int rows;
+    int d;
+    float* out;
+};
+cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, int32_t* device_status, cudaStream_t stream);
 
 }  // namespace polyspec

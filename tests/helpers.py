@@ -173,3 +173,16 @@ def compare_level_batch(gpu_a, gpu_next, ora, seqs=None, band=TIE_BAND):
         if kind == "mismatch":
             bad.append((b, int(gpu_a[b]), int(gpu_next[b]), int(ora["accepted_len"][b]), int(ora["next_token"][b])))
     return counts, bad
+
+
+def cdf_distance(weights, u, token):
+    """Distance, in normalised CDF units, from the uniform u to the inverse-CDF interval of `token`
+    under the (unnormalised, float64) weights; 0 if u falls inside it.  inf for a zero-mass token."""
+    w = np.asarray(weights, dtype=np.float64)
+    if token < 0 or token >= len(w) or not (w[token] > 0.0):
+        return float("inf")
+    c = np.cumsum(w)
+    total = c[-1]
+    lo = (c[token] - w[token]) / total
+    hi = c[token] / total
+    return float(max(lo - u, u - hi, 0.0))
