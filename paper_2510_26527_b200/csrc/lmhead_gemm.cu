@@ -2,26 +2,36 @@
 // (the last op of the model forwards in Algorithm 1, "p_{1:K} <- M_2(...)" and
 // "v <- M_1(...)"), bf16 inputs, fp32 accumulation, fp32 logits out.
 //
-// The contraction is dense, so it runs on tcgen05: the vocabulary is the MMA's M axis (a
-// CTA owns 128 vocabulary entries at a time), the (sequence, position) rows of the hidden
-// states are the N axis (up to 288 columns per accumulator, issued as one or two MMAs of
-// N <= 256), and d is the K loop in blocks of 64 elements = one 128-byte swizzle row.
-// Both operands are K-major in shared memory exactly as 2-D TMA with 128-byte swizzle
-// writes them.  The accumulator lives in TMEM (lane = vocabulary entry, column = hidden
-// row) and is read back with tcgen05.ld by four epilogue warps.
+// The contraction is dense, so it runs on tcgen05.  It is also skinny (a few hundred hidden
+// rows against the whole vocabulary), which makes it a weight-streaming problem: per flop it
+// needs more shared-memory fill than a square GEMM, and W arrives at HBM latency.  Hence:
+//   - the vocabulary is the MMA's M axis and two CTAs on neighbouring SMs work as a pair
+//     (cta_group::2, M = 256): each CTA streams its own 128 rows of W, and the hidden tile
+//     (the N axis, up to 288 columns, one or two MMAs of N <= 256) is split between the two,
+//     so each SM fills and reads only half of it;
+//   - d is the K loop in blocks of 64 elements = one 128-byte swizzle row; both operands are
+//     K-major in shared memory exactly as 2-D TMA with 128-byte swizzle writes them; a
+//     6-stage ring of (W tile, hidden half-tile) keeps about 200 KiB in flight per SM;
+//   - the accumulator lives in TMEM (lane = vocabulary entry, column = hidden row) and is
+//     read back with tcgen05.ld by four epilogue warps per CTA.
 //
-// One persistent CTA per SM walks a static list of work items (model, vocabulary tile,
-// column block), costliest model first, so the target's and the drafter's projections
-// share one launch and the tail of one fills the other's idle SMs.  Warp roles:
-//   warp 0      TMA producer (one lane): W tile + hidden tile per K block into a 4-stage ring
-//   warp 1      MMA issuer (one lane); also allocates / frees TMEM
-//   warps 2..5  epilogue: TMEM -> registers -> global, 128-byte coalesced stores per column
+// The grid is persistent: CTA pair i walks work items i, i + pairs, ... of a static list
+// (model, 256-entry vocabulary tile, column block), costliest model first, so the target's and
+// the drafter's projections share one launch and the tail of one fills the other's idle SMs.
+// Warp roles in each CTA:
+//   warp 0      TMA producer (one elected lane issues).  Both CTAs load their own tiles; all copies of a stage
+//               complete on the leader CTA's "full" barrier (no multicast anywhere)
+//   warp 6      L2 prefetch of W: 1 KiB contiguous per row, a few K blocks ahead of the TMA loads
+//   warp 1      MMA issuer (one elected lane, leader CTA only); allocates / frees TMEM in both CTAs.
+//               tcgen05.commit arrives on the "empty" / "accumulator full" barriers of both CTAs
+//   warps 2..5  epilogue: TMEM -> registers -> global, 128-byte coalesced stores per column; all
+//               eight epilogue warps of the pair arrive on the leader's "accumulator empty" barrier
 // When a column block needs at most 256 TMEM columns two accumulators alternate, so the
 // epilogue of one tile overlaps the K loop of the next.
 //
-// Every wait is bounded.  A wait that runs out raises an abort flag that all roles poll,
-// sets POLYSPEC_ERR_TIMEOUT in the status word, lets copies and MMAs in flight finish
-// (bounded again), frees TMEM and returns.
+// Every wait on an mbarrier is bounded.  A wait that runs out raises an abort flag in both CTAs
+// that all roles poll, sets POLYSPEC_ERR_TIMEOUT in the status word, lets copies in flight land
+// (bounded again), and the kernel still frees TMEM and returns.
 #include <cuda.h>
 
 #include "polyspec_kernels.cuh"
@@ -29,27 +39,31 @@
 namespace polyspec {
 namespace {
 
-constexpr int kTileV = 128;                 // vocabulary entries per tile (MMA M)
+constexpr int kTileV = 128;                 // vocabulary entries per CTA and tile (MMA M per CTA)
+constexpr int kPairV = 2 * kTileV;          // vocabulary entries per CTA pair and tile (MMA M)
 constexpr int kBlockK = 64;                 // bf16 elements per K block (one 128-byte swizzle row)
 constexpr int kMmaK = 16;                   // K of one tcgen05.mma for 16-bit inputs
 constexpr int kMaxCols = 288;               // widest column block (TMEM columns per accumulator)
-constexpr int kStagesG = 4;
-constexpr int kBytesA = kTileV * kBlockK * 2;          // 16 KiB
-constexpr int kBytesBMax = kMaxCols * kBlockK * 2;     // 36 KiB
-constexpr int kStageBytes = kBytesA + kBytesBMax;
-constexpr int kGemmThreads = 192;
+constexpr int kStagesG = 6;
+constexpr int kBytesA = kTileV * kBlockK * 2;                // 16 KiB: this CTA's rows of W
+constexpr int kBytesBMax = (kMaxCols / 2) * kBlockK * 2;     // 18 KiB: this CTA's half of the hidden tile
+constexpr int kStageBytes = kBytesA + kBytesBMax;            // 34 KiB
+constexpr int kGemmThreads = 224;
+constexpr int kPrefetchK = 8;               // K blocks per L2 prefetch: 1 KiB contiguous per W row
+constexpr int kPrefetchLead = 16;           // how many K blocks the prefetch may run ahead of the TMA loads
 constexpr int kTmemCols = 512;
-constexpr uint32_t kSpinLimitG = 1u << 22;
+constexpr uint32_t kSpinLimitG = 1u << 20;
 constexpr size_t kGemmSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStagesG) * kStageBytes + 256 /* barriers */;
 
 struct GemmJob {
     CUtensorMap map_w;      // [V, d] bf16, box {64, 128}
-    CUtensorMap map_h;      // [rows, d] bf16, box {64, chunk}
+    CUtensorMap map_h;      // [rows, d] bf16, box {64, chunk / 2}
+    const char* w;          // W itself, for the L2 prefetch that runs ahead of the TMA loads
     float* out;             // [rows, V]
     int rows;
     int kblocks;            // d / 64
     int block_cols;         // columns (hidden rows) per work item, multiple of 16, <= 288
-    int chunk;              // columns per MMA / per hidden TMA box, multiple of 16, <= 256
+    int chunk;              // columns per MMA, multiple of 16, <= 256; each CTA holds chunk / 2 of them
     int nchunks;            // block_cols / chunk
     int nblocks;            // column blocks covering `rows`
     int items;              // vocabulary tiles * nblocks
@@ -59,13 +73,32 @@ struct GemmParams {
     GemmJob job[2];
     int n_jobs;
     int V;
-    int vtiles;
+    int vtiles;             // 256-entry vocabulary tiles
     int total_items;
     int acc_stages;         // 2 when every job's column block fits 256 TMEM columns (accumulators at columns 0 and 256), else 1
     int32_t* status;
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+// The shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
@@ -75,9 +108,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+// Arrive on a barrier of any CTA of the cluster (`bar` is a shared::cluster address).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar)
 {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
 {
@@ -89,7 +123,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait that also gives up when another role has raised the abort flag.
+// Bounded wait that also gives up when a role of either CTA has raised the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
     for (uint32_t i = 0; i < kSpinLimitG; ++i) {
@@ -99,40 +133,59 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// 2-D tiled TMA load into this CTA's shared memory; completion is counted on `bar`, a
+// shared::cluster address that may belong to the peer CTA of the pair.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
-// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes with the
-// 128-byte swizzle: 8-row groups 1024 bytes apart (stride byte offset), descriptor
-// version 1, layout type 2.  `addr` may point 32 * i bytes into the first row to select
-// the i-th 16-element K slice.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
-{
-    return static_cast<uint64_t>((addr & 0x3ffffu) >> 4) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
-}
-
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+// Shared-memory matrix descriptor (64 bits) of a K-major tile stored as rows of 128 bytes with
+// the 128-byte swizzle: start address >> 4 in bits 0..13, leading byte offset (unused here, 1) in
+// bits 16..29, stride byte offset 1024 >> 4 (8-row groups 1024 bytes apart) in bits 32..45,
+// descriptor version 1 in bits 46..47, layout type 2 in bits 61..63.  The address may point
+// 32 * i bytes into the first row to select the i-th 16-element K slice.
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 256 over the CTA pair, N = n.
 __device__ __forceinline__ uint32_t instr_desc_bf16(int n)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileV >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kPairV >> 4) << 24);
 }
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+// The upper word of smem_desc_sw128 is the same for every tile; MMAs are issued from the lower words.
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t addr) { return ((addr & 0x3ffffu) >> 4) | (1u << 16); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t adesc_lo, uint32_t bdesc_lo, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(adesc_lo), "r"(bdesc_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
 }
-__device__ __forceinline__ void umma_commit(uint32_t bar)
+// Arrives (once all MMAs issued so far have completed) on the barrier at offset `bar` in both CTAs.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    const unsigned short mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+// True in exactly one lane of a fully active warp.  The role loops are run by whole warps
+// (every lane polls the barriers) and only the issue of an asynchronous instruction is
+// elected, so that loop state and descriptors stay warp-uniform.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -160,124 +213,183 @@ __device__ __forceinline__ void decode_item(const GemmParams& p, int item, int* 
     *nb = item - (item / nbk) * nbk;
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1) lmhead_kernel(const __grid_constant__ GemmParams p)
+// Sets the abort flag of both CTAs of the pair and records the timeout.
+__device__ __forceinline__ void raise_abort(int* abort_flag, uint32_t peer, int32_t* status)
+{
+    if (!*reinterpret_cast<volatile int*>(abort_flag) && status) atomicCAS(status, 0, static_cast<int>(POLYSPEC_ERR_TIMEOUT));
+    *reinterpret_cast<volatile int*>(abort_flag) = 1;
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr(smem_addr(abort_flag), peer)), "r"(1) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmhead_kernel(const __grid_constant__ GemmParams p)
 {
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ uint32_t loads_issued;       // K blocks the TMA producer has issued so far
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // 128-byte swizzled tiles must start on a 1024-byte boundary
+    // broadcast from lane 0 so that the compiler knows the role branches and everything derived
+    // from them (ring positions, descriptors) are warp-uniform
+    const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();           // 0 = leader of the pair
+    const uint32_t peer = rank ^ 1u;
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    // 128-byte swizzled tiles must start on a 1024-byte boundary; both CTAs use the same offsets
     const uint32_t raw = smem_addr(smem_dyn);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
-    const uint32_t bars = tiles + kStagesG * kStageBytes;      // full[4], empty[4], acc_full[2], acc_empty[2]
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (kStagesG + s); };
-    auto accf_bar = [&](int a) { return bars + 8u * (2 * kStagesG + a); };
-    auto acce_bar = [&](int a) { return bars + 8u * (2 * kStagesG + 2 + a); };
+    const uint32_t bars = tiles + kStagesG * kStageBytes;
+    const uint32_t full_bar = bars, empty_bar = full_bar + 8u * kStagesG;       // full: used in the leader only
+    const uint32_t acc_full = empty_bar + 8u * kStagesG, acc_empty = acc_full + 16u;   // acc_empty: leader only
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(accf_bar(a), 1); mbar_init(acce_bar(a), 4); }
+        loads_issued = 0;
+        for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full + 8u * a, 1); mbar_init(acc_empty + 8u * a, 8); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base_slot)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();             // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abort_p = &abort_flag;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t it = 0;          // K blocks issued so far (ring position)
-            bool ok = true;
-            for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x) {
-                int j, vt, nb;
-                decode_item(p, item, &j, &vt, &nb);
-                const GemmJob& job = p.job[j];
-                const uint32_t bytes = kBytesA + static_cast<uint32_t>(job.block_cols) * kBlockK * 2;
-                for (int kb = 0; kb < job.kblocks; ++kb, ++it) {
-                    const int s = it % kStagesG;
-                    if (!mbar_wait(empty_bar(s), ((it / kStagesG) & 1u) ^ 1u, abort_p)) { ok = false; break; }
-                    mbar_expect_tx(full_bar(s), bytes);
-                    const uint32_t a_dst = tiles + s * kStageBytes;
-                    tma_load_2d(a_dst, &job.map_w, kb * kBlockK, vt * kTileV, full_bar(s));
-                    for (int c = 0; c < job.nchunks; ++c)
-                        tma_load_2d(a_dst + kBytesA + c * job.chunk * (kBlockK * 2), &job.map_h, kb * kBlockK,
-                                    nb * job.block_cols + c * job.chunk, full_bar(s));
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        uint32_t it = 0;          // K blocks issued so far
+        uint32_t stage = 0, phase = 1;      // ring position; a fresh "empty" barrier passes a wait on parity 1
+        bool ok = true;
+        const uint32_t leader_full = cluster_addr(full_bar, 0);
+        for (int item = pair; ok && item < p.total_items; item += n_pairs) {
+            int j, vt, nb;
+            decode_item(p, item, &j, &vt, &nb);
+            const GemmJob& job = p.job[j];
+            const int half = job.chunk >> 1;
+            const uint32_t pair_bytes = 2u * (kBytesA + static_cast<uint32_t>(job.block_cols >> 1) * (kBlockK * 2));
+            const int w_row = vt * kPairV + static_cast<int>(rank) * kTileV;
+            const int h_row = nb * job.block_cols + static_cast<int>(rank) * half;
+            const bool two = job.nchunks == 2;
+            for (int kb = 0; kb < job.kblocks; ++kb, ++it) {
+                if (!mbar_wait(empty_bar + 8u * stage, phase, abort_p)) { ok = false; break; }
+                const uint32_t bar = leader_full + 8u * stage;
+                const uint32_t a_dst = tiles + stage * kStageBytes;
+                if (elect_one()) {
+                    if (rank == 0) mbar_expect_tx(full_bar + 8u * stage, pair_bytes);
+                    tma_load_2d(a_dst, &job.map_w, kb * kBlockK, w_row, bar);
+                    tma_load_2d(a_dst + kBytesA, &job.map_h, kb * kBlockK, h_row, bar);
+                    if (two) tma_load_2d(a_dst + kBytesA + half * (kBlockK * 2), &job.map_h, kb * kBlockK, h_row + job.chunk, bar);
+                    *reinterpret_cast<volatile uint32_t*>(&loads_issued) = it + 1;
                 }
+                __syncwarp();
+                if (++stage == kStagesG) { stage = 0; phase ^= 1u; }
             }
-            if (!ok) {
-                if (!*abort_p && p.status) atomicCAS(p.status, 0, static_cast<int>(POLYSPEC_ERR_TIMEOUT));
-                *abort_p = 1;
-            }
-            // copies still in flight must land before the CTA may exit: the last kStagesG fills
-            const uint32_t first = it > static_cast<uint32_t>(kStagesG) ? it - kStagesG : 0u;
-            for (uint32_t q = first; q < it; ++q) {
-                const int s = q % kStagesG;
-                for (uint32_t i = 0; i < kSpinLimitG; ++i)
-                    if (mbar_try(full_bar(s), (q / kStagesG) & 1u)) break;
+        }
+        if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
+        __syncwarp();
+        // this CTA's copies must have landed before it may exit.  The leader sees them on its own
+        // "full" barriers; the peer learns it from the leader's commits on its "empty" barriers,
+        // which follow the MMAs that read the stage.
+        const uint32_t first = it > static_cast<uint32_t>(kStagesG) ? it - kStagesG : 0u;
+        for (uint32_t q = first; q < it; ++q) {
+            const uint32_t b = (rank == 0 ? full_bar : empty_bar) + 8u * (q % kStagesG);
+            for (uint32_t i = 0; i < kSpinLimitG; ++i)
+                if (mbar_try(b, (q / kStagesG) & 1u) || *abort_p) break;
+        }
+    } else if (warp == 6) {
+        // ------------------------------------------------------------------ L2 prefetch of W (both CTAs)
+        // A TMA box touches 128 bytes in each of 128 rows of W that lie d * 2 bytes apart: 128 DRAM
+        // pages per K block, each page visited again only a K block later.  This warp runs a little
+        // ahead and asks L2 for 1 KiB contiguous per row (8 K blocks at once), so DRAM sees page-long
+        // bursts and the TMA loads find their lines in L2.
+        uint32_t it = 0;
+        bool live = true;
+        for (int item = pair; live && item < p.total_items; item += n_pairs) {
+            int j, vt, nb;
+            decode_item(p, item, &j, &vt, &nb);
+            const GemmJob& job = p.job[j];
+            const size_t row_bytes = static_cast<size_t>(job.kblocks) * (kBlockK * 2);
+            const int v0 = vt * kPairV + static_cast<int>(rank) * kTileV;
+            for (int kb = 0; live && kb < job.kblocks; kb += kPrefetchK) {
+                uint32_t spins = 0;
+                while (*reinterpret_cast<volatile uint32_t*>(&loads_issued) + kPrefetchLead < it) {
+                    __nanosleep(64);
+                    if (*abort_p || ++spins > (1u << 22)) { live = false; break; }
+                }
+                if (!live) break;
+                const int nk = min(kPrefetchK, job.kblocks - kb);
+                it += nk;
+#pragma unroll
+                for (int q = 0; q < kTileV / 32; ++q) {
+                    const int v = v0 + q * 32 + lane;
+                    if (v < p.V) {
+                        const char* src = job.w + static_cast<size_t>(v) * row_bytes + static_cast<size_t>(kb) * (kBlockK * 2);
+                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(nk * kBlockK * 2) : "memory");
+                    }
+                }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            uint32_t it = 0, tile_n = 0;
+        // ------------------------------------------------------------------ MMA issuer (leader CTA)
+        if (rank == 0) {
+            uint32_t stage = 0, phase = 0, tile_n = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x, ++tile_n) {
+            for (int item = pair; ok && item < p.total_items; item += n_pairs, ++tile_n) {
                 int j, vt, nb;
                 decode_item(p, item, &j, &vt, &nb);
                 const GemmJob& job = p.job[j];
                 const int acc = tile_n % p.acc_stages;
                 const uint32_t use = tile_n / p.acc_stages;        // how often this accumulator was used before
-                if (!mbar_wait(acce_bar(acc), (use & 1u) ^ 1u, abort_p)) { ok = false; break; }
+                if (!mbar_wait(acc_empty + 8u * acc, (use & 1u) ^ 1u, abort_p)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t idesc = instr_desc_bf16(job.chunk);
                 const uint32_t d_tmem = tmem_base + acc * (kTmemCols / 2);
-                for (int kb = 0; kb < job.kblocks; ++kb, ++it) {
-                    const int s = it % kStagesG;
-                    if (!mbar_wait(full_bar(s), (it / kStagesG) & 1u, abort_p)) { ok = false; break; }
+                const uint32_t b_chunk = static_cast<uint32_t>(job.chunk >> 1) * (kBlockK * 2) >> 4;   // second MMA's B tile, in 16-byte units
+                const bool two = job.nchunks == 2;
+                for (int kb = 0; kb < job.kblocks; ++kb) {
+                    if (!mbar_wait(full_bar + 8u * stage, phase, abort_p)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = tiles + s * kStageBytes;
-                    const uint32_t b_addr = a_addr + kBytesA;
+                    const uint32_t a_lo = smem_desc_lo(tiles + stage * kStageBytes);
+                    const uint32_t b_lo = a_lo + (kBytesA >> 4);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < kBlockK / kMmaK; ++kk) {
-                        const uint64_t adesc = smem_desc_sw128(a_addr + kk * (kMmaK * 2));
-                        for (int c = 0; c < job.nchunks; ++c) {
-                            const uint64_t bdesc = smem_desc_sw128(b_addr + c * job.chunk * (kBlockK * 2) + kk * (kMmaK * 2));
-                            umma_bf16(d_tmem + c * job.chunk, adesc, bdesc, idesc, (kb | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < kBlockK / kMmaK; ++kk) {
+                            const uint32_t acc_flag = (kb | kk) != 0 ? 1u : 0u;
+                            umma_bf16(d_tmem, a_lo + kk * (kMmaK * 2 >> 4), b_lo + kk * (kMmaK * 2 >> 4), idesc, acc_flag);
+                            if (two)
+                                umma_bf16(d_tmem + job.chunk, a_lo + kk * (kMmaK * 2 >> 4), b_lo + b_chunk + kk * (kMmaK * 2 >> 4), idesc, acc_flag);
                         }
+                        umma_commit_pair(empty_bar + 8u * stage);      // frees the stage in both CTAs once these MMAs have read it
                     }
-                    umma_commit(empty_bar(s));          // frees the stage once these MMAs have read it
+                    __syncwarp();
+                    if (++stage == kStagesG) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) umma_commit(accf_bar(acc));     // accumulator complete
+                if (ok && elect_one()) umma_commit_pair(acc_full + 8u * acc);     // accumulator complete, in both CTAs
+                __syncwarp();
             }
-            if (!ok) {
-                if (!*abort_p && p.status) atomicCAS(p.status, 0, static_cast<int>(POLYSPEC_ERR_TIMEOUT));
-                *abort_p = 1;
-            }
+            if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
+            __syncwarp();
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
         const int quarter = warp & 3;                   // the TMEM lanes this warp may read: 32 * quarter ..
+        const uint32_t leader_acc_empty = cluster_addr(acc_empty, 0);
         uint32_t tile_n = 0;
         bool ok = true;
-        for (int item = blockIdx.x; ok && item < p.total_items; item += gridDim.x, ++tile_n) {
+        for (int item = pair; ok && item < p.total_items; item += n_pairs, ++tile_n) {
             int j, vt, nb;
             decode_item(p, item, &j, &vt, &nb);
             const GemmJob& job = p.job[j];
             const int acc = tile_n % p.acc_stages;
             const uint32_t use = tile_n / p.acc_stages;
-            if (!mbar_wait(accf_bar(acc), use & 1u, abort_p)) { ok = false; break; }
+            if (!mbar_wait(acc_full + 8u * acc, use & 1u, abort_p)) { ok = false; break; }
             tc_fence_after();
-            const int v = vt * kTileV + quarter * 32 + lane;
+            const int v = vt * kPairV + static_cast<int>(rank) * kTileV + quarter * 32 + lane;
             const int row0 = nb * job.block_cols;
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * (kTmemCols / 2);
             float* out_v = job.out + v;
@@ -295,23 +407,22 @@ __global__ void __launch_bounds__(kGemmThreads, 1) lmhead_kernel(const __grid_co
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce_bar(acc));
+            if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8u * acc);
         }
-        if (!ok && lane == 0) {
-            if (!*abort_p && p.status) atomicCAS(p.status, 0, static_cast<int>(POLYSPEC_ERR_TIMEOUT));
-            *abort_p = 1;
-        }
+        if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
     }
 
+    // Neither CTA may leave (or free TMEM) while the other can still signal its barriers or while
+    // MMAs of the pair are in flight: in the normal course every MMA has been waited for through
+    // the accumulator barriers by the time the epilogues are done.
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     tc_fence_after();
     if (warp == 1) {
-        // every MMA this CTA issued has been waited for through the accumulator barriers unless the
-        // kernel is aborting; in that case give the tensor core a bounded moment before freeing TMEM
-        if (*abort_p) __nanosleep(1000000);
+        if (*abort_p) __nanosleep(1000000);      // aborting: give MMAs in flight a bounded moment
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -321,7 +432,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 EncodeTiledFn g_encode = nullptr;
 bool g_attr_set[64] = {false};
-int g_sms[64] = {0};
+int g_pairs[64] = {0};      // CTA pairs the device can hold at once
 
 cudaError_t get_encoder()
 {
@@ -365,14 +476,30 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, int32_t* dev
         int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        g_sms[dev] = sms > 0 ? sms : 148;
+        if (sms <= 0) sms = 148;
+        // how many 2-CTA clusters fit at once (an odd SM of a GPC cannot host one)
+        int clusters = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(sms / 2 * 2));
+        cfg.blockDim = dim3(kGemmThreads);
+        cfg.dynamicSmemBytes = kGemmSmemBytes;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaOccupancyMaxActiveClusters(&clusters, lmhead_kernel, &cfg) != cudaSuccess || clusters <= 0) {
+            (void)cudaGetLastError();
+            clusters = sms / 2;
+        }
+        g_pairs[dev] = clusters < sms / 2 ? clusters : sms / 2;
         g_attr_set[dev] = true;
     }
 
     GemmParams p;
     p.n_jobs = n;
     p.V = V;
-    p.vtiles = (V + kTileV - 1) / kTileV;
+    p.vtiles = (V + kPairV - 1) / kPairV;
     p.status = device_status;
     p.total_items = 0;
     p.acc_stages = 2;
@@ -396,14 +523,15 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, int32_t* dev
         job.rows = pr.rows;
         job.kblocks = pr.d / kBlockK;
         job.out = pr.out;
+        job.w = static_cast<const char*>(pr.W);
         job.items = p.vtiles * job.nblocks;
         p.total_items += job.items;
         if (cols > kTmemCols / 2) p.acc_stages = 1;
         if (!encode_map(&job.map_w, pr.W, V, pr.d, kTileV)) return cudaErrorInvalidValue;
-        if (!encode_map(&job.map_h, pr.hidden, pr.rows, pr.d, job.chunk)) return cudaErrorInvalidValue;
+        if (!encode_map(&job.map_h, pr.hidden, pr.rows, pr.d, job.chunk / 2)) return cudaErrorInvalidValue;
     }
-    const int grid = p.total_items < g_sms[dev] ? p.total_items : g_sms[dev];
-    lmhead_kernel<<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(p);
+    const int pairs = p.total_items < g_pairs[dev] ? p.total_items : g_pairs[dev];
+    lmhead_kernel<<<2 * pairs, kGemmThreads, kGemmSmemBytes, stream>>>(p);
     return cudaGetLastError();
 }
 
