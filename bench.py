@@ -3,6 +3,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2|cfg1|cfg4] [--impl reference]
 
+`--workload cfg4` is the fused path (hidden states -> LM-head projections on the tensor cores -> verification); its
+roofline object is the tensor one.
+
 One step = one pass of the whole hot path (row statistics over every logits row of every model,
 then accept tests / first rejection / replacement-or-bonus sampling / hand-off for every level)
 over one batch that is already resident in HBM.  The default workload is the largest logits-path
@@ -37,7 +40,9 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-statistics kernel, from the ncu
 # capture summarised under profiles/ (bytes per logits byte processed, measured on a smaller case of
 # the same kernel and scaled by the bytes one launch processes).  None until a capture exists.
-STATS_TRAFFIC_PER_LOGIT_BYTE = None
+STATS_TRAFFIC_PER_LOGIT_BYTE = 1.0156     # profiles/stats_kernel_bf16_cfg3_ncu_full.md: (328.362 + 5.106) MB moved for 328.340 MB of logits
+# the same counters per launch of the LM-head kernel on the fused workload (profiles/); None until captured
+LMHEAD_TRAFFIC_BYTES = None
 
 
 def read_peaks():
@@ -127,25 +132,45 @@ def oracle_time(sample, threads):
 
 
 def cpu_baseline(data, spec, target_seconds=12.0):
-    """The oracle, as it stands, on the first sequences of the resident batch: about target_seconds of CPU work."""
+    """The oracle, as it stands, on the resident batch: whole passes over it until about target_seconds of CPU work."""
     from oracle import oracle as orc
     orc.build()
     cores = os.cpu_count() or 1
-    B = spec.B
-
-    def take(n):
-        return {"models": [m[:n].cpu() for m in data["models"]], "k": data["k"],
-                "draft_tokens": data["draft_tokens"][:n].cpu(), "uniforms": data["uniforms"][:, :n].cpu().contiguous(),
-                "temperature": data["temperature"]}
-    n0 = min(B, cores)
-    tok0, t0 = oracle_time(take(n0), cores)
-    n = int(min(B, max(n0, n0 * target_seconds / max(t0, 1e-3))))
-    n = max(cores, n // cores * cores) if n >= cores else n
-    n = min(n, B)
-    tok, t = oracle_time(take(n), cores)
+    sample = {"models": [m.cpu() for m in data["models"]], "k": data["k"], "draft_tokens": data["draft_tokens"].cpu(),
+              "uniforms": data["uniforms"].cpu().contiguous(), "temperature": data["temperature"]}
+    tok0, t0 = oracle_time(sample, cores)
+    passes = int(min(200, max(1, round(target_seconds / max(t0, 1e-3)))))
+    tok, t = 0, 0.0
+    for _ in range(passes):
+        a, b = oracle_time(sample, cores)
+        tok += a
+        t += b
     return {"value": tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n} of {B} sequences of the same batch, {tok} verified tokens in {t:.2f} s, "
+            "sample": f"{passes} passes over the {spec.B} sequences of the same batch, {tok} verified tokens in {t:.2f} s, "
                       f"{cores} threads (one sequence per thread)"}
+
+
+def fused_oracle_time(d, n_seq, threads):
+    from oracle import oracle as orc
+    t0 = time.perf_counter()
+    out = orc.verify_from_hidden(d["hidden_p"][:n_seq], d["W_p"], d["hidden_q"][:n_seq], d["W_q"], d["draft_tokens"][:n_seq].cpu(),
+                                 d["uniforms"][:n_seq].cpu(), d["temperature"], threads=threads)
+    dt = time.perf_counter() - t0
+    return int(n_seq * d["draft_tokens"].shape[1]), dt, out
+
+
+def fused_cpu_baseline(d, spec, target_seconds=12.0):
+    """The oracle's float64 projection + verification on the first sequences of the batch."""
+    from oracle import oracle as orc
+    orc.build()
+    cores = os.cpu_count() or 1
+    n0 = min(spec.B, 2)
+    tok0, t0, _ = fused_oracle_time(d, n0, cores)
+    n = int(min(spec.B, max(n0, n0 * target_seconds / max(t0, 1e-3))))
+    tok, t, _ = fused_oracle_time(d, n, cores)
+    return {"value": tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {spec.B} sequences of the same batch (float64 matmul of the LM head on the host, then the "
+                      f"verification rule), {tok} verified tokens in {t:.2f} s, {cores} threads"}
 
 
 def run_reference(args, spec):
@@ -157,13 +182,20 @@ def run_reference(args, spec):
     orc.build()
     cores = os.cpu_count() or 1
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
-    n_seq = min(spec.B, 8 * cores)
-    sample = oracle_sample(spec, seed=args.seed, n_seq=n_seq, device=dev)
+    if isinstance(spec, synth.FusedSpec):
+        n_seq = min(spec.B, 4)
+        d = synth.make_fused(spec, seed=args.seed, device=dev)
+        d = {k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}
+        step = lambda: fused_oracle_time(d, n_seq, cores)[:2]
+    else:
+        n_seq = min(spec.B, 8 * cores)
+        sample = oracle_sample(spec, seed=args.seed, n_seq=n_seq, device=dev)
+        step = lambda: oracle_time(sample, cores)
     for _ in range(args.warmup):
-        oracle_time(sample, cores)
+        step()
     tokens, elapsed = 0, 0.0
     for _ in range(args.steps):
-        tok, dt = oracle_time(sample, cores)
+        tok, dt = step()
         tokens += tok
         elapsed += dt
     value = tokens / elapsed
@@ -180,6 +212,9 @@ def run_reference(args, spec):
 
 
 def workload_name(args, spec):
+    if isinstance(spec, synth.FusedSpec):
+        return (f"cfg4: fused LM-head verify, B={spec.B} per GPU, k={spec.k}, V={spec.V}, hidden bf16 [{spec.B},{spec.k + 1},{spec.d_p}] / "
+                f"[{spec.B},{spec.rows_q},{spec.d_q}], LM-head weights bf16 [{spec.V},{spec.d_p}] / [{spec.V},{spec.d_q}], T={spec.temperature}")
     k_bottom_up = tuple(reversed(spec.k))
     extra = f", inter-level sigma {args.sigma}" if spec.name == "cfg5" else ""
     return (f"{spec.name}: {spec.n_models}-level chain, B={spec.B} per GPU, V={spec.V}, "
@@ -318,22 +353,152 @@ def run_gpu(args, spec):
         dist.destroy_process_group()
 
 
+def run_gpu_fused(args, spec):
+    """cfg4: hidden states -> LM-head projections on the tensor cores -> verification, one C-ABI call per step."""
+    from paper_2510_26527_b200 import binding, buildlib
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: libpolyspec has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        buildlib.build()
+    if world > 1:
+        dist.barrier()
+    binding.load_library()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    d = synth.make_fused(spec, seed=args.seed + 7919 * rank, device=dev)
+    call = binding.FusedCall(d["hidden_p"], d["W_p"], d["hidden_q"], d["W_q"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    for _ in range(max(args.warmup, 3)):
+        call.launch()
+    torch.cuda.synchronize()
+    assert int(call.device_status.item()) == 0
+    tokens_per_step = spec.B * spec.k
+    emitted_per_step = int((call.out["accepted_len"] + 1).sum().item())
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        call.project()
+        ev[i][1].record()
+        call.verify()
+        ev[i][2].record()
+    stop.record()
+    barrier()
+    elapsed_ms = start.elapsed_time(stop)
+    clocks = sampler.stop() if rank == 0 else None
+    gemm_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
+    verify_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+
+    # end to end: this step's hidden states, draft tokens and uniforms come from pinned host memory, the
+    # outputs go back to pinned host memory; the LM-head weights are model parameters and stay resident
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_in = [t.cpu().pin_memory() for t in (d["hidden_p"], d["hidden_q"], d["draft_tokens"], d["uniforms"])]
+    dev_in = [d["hidden_p"], d["hidden_q"], d["draft_tokens"], d["uniforms"]]
+    host_out = [torch.empty(spec.B, dtype=torch.int32).pin_memory() for _ in range(2)]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = 2 * spec.B * 4
+
+    def e2e_step():
+        for h, g in zip(host_in, dev_in):
+            g.copy_(h, non_blocking=True)
+        call.launch()
+        host_out[0].copy_(call.out["accepted_len"], non_blocking=True)
+        host_out[1].copy_(call.out["next_token"], non_blocking=True)
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([elapsed_ms, e2e_ms, gemm_ms, verify_ms], device=dev, dtype=torch.float64)
+    w = torch.tensor([tokens_per_step, emitted_per_step], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    elapsed_ms, e2e_ms, gemm_ms, verify_ms = (float(x) for x in t.tolist())
+    tokens_all, emitted_all = (float(x) for x in w.tolist())
+
+    base = None
+    if rank == 0 and not args.no_cpu_baseline:
+        base = fused_cpu_baseline({k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}, spec, target_seconds=args.cpu_seconds)
+
+    if rank == 0:
+        peaks = read_peaks()
+        ms_per_step = elapsed_ms / args.steps
+        flops = spec.flops()
+        achieved = flops / (gemm_ms * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": tokens_all * args.steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(args, spec), "seed": args.seed,
+                       "l2": f"inputs {(spec.weight_bytes() + 2 * spec.B * (spec.k + 1) * (spec.d_p + spec.d_q)) / 1e9:.3f} GB per step, "
+                             "larger than the 126 MB L2; no flush needed",
+                       "parallelism": f"{world} independent replicas, batch sharded, no collective"},
+            "gpu_launches": 3 * args.steps,
+            "emitted_tokens_per_s": emitted_all * args.steps / (elapsed_ms * 1e-3),
+            "whole_step_tflops": flops * world / (ms_per_step * 1e-3) / 1e12,
+            "whole_step_frac_of_tensor_peak": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "kernel_ms": {"lm_head_project": gemm_ms, "row_stats_and_walk": verify_ms},
+            "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (both LM-head projections, tcgen05 cta_group::2)",
+                         "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                         "traffic": LMHEAD_TRAFFIC_BYTES, "peak_source": f"of {peaks['source']} (burst)",
+                         "weight_stream_gbs": spec.weight_bytes() / (gemm_ms * 1e-3) / 1e9,
+                         "weight_stream_frac_of_hbm_peak": spec.weight_bytes() / (gemm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "e2e": {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                    "note": "hidden states, tokens and uniforms copied per step; LM-head weights resident"},
+            "clocks": clocks,
+        }
+        if base is not None:
+            line["cpu_baseline"] = base
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="polyspec", choices=["polyspec", "reference"])
-    ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg5"])
+    ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--sigma", type=float, default=1.0, help="inter-level noise of cfg5")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    spec = chain_spec(args.workload, args.sigma)
+    spec = synth.FusedSpec() if args.workload == "cfg4" else chain_spec(args.workload, args.sigma)
     if args.impl == "reference":
         run_reference(args, spec)
+    elif args.workload == "cfg4":
+        run_gpu_fused(args, spec)
     else:
         run_gpu(args, spec)
 

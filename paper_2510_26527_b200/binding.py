@@ -28,6 +28,7 @@ EXPORTS = (
     "polyspec_chain_row_stats", "polyspec_chain_walk",
     "polyspec_verify_chain_host_workspace", "polyspec_verify_chain_host",
     "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden", "polyspec_lm_head",
+    "polyspec_from_hidden_project", "polyspec_from_hidden_verify",
     "polyspec_static_scratch_bytes", "polyspec_verify_level_static",
 )
 
@@ -85,6 +86,10 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_from_hidden.restype = ci
     lib.polyspec_verify_from_hidden.argtypes = [vp, vp, vp, vp, ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf,
                                                 i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
+    lib.polyspec_from_hidden_project.restype = ci
+    lib.polyspec_from_hidden_project.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, i32p, vp, sz, vp]
+    lib.polyspec_from_hidden_verify.restype = ci
+    lib.polyspec_from_hidden_verify.argtypes = [ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf, i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
     lib.polyspec_lm_head.restype = ci
     lib.polyspec_lm_head.argtypes = [vp, vp, ci, ci, ci, f32p, i32p, vp]
     lib.polyspec_static_scratch_bytes.restype = sz
@@ -360,6 +365,59 @@ def polyspec_verify_from_hidden(hidden_p, W_p, hidden_q, W_q, draft_tokens, unif
     _check(st, "polyspec_verify_from_hidden")
     out["device_status"] = device_status
     return out
+
+
+class FusedCall:
+    """A prepared polyspec_verify_from_hidden call: arguments marshalled once, outputs and workspace allocated once.
+
+    launch() is the single C-ABI call; project() and verify() are its two halves
+    (polyspec_from_hidden_project / polyspec_from_hidden_verify)."""
+
+    def __init__(self, hidden_p, W_p, hidden_q, W_q, draft_tokens, uniforms, temperature, block_len=None, stream=None):
+        self.lib = load_library()
+        _dev_check(hidden_p, W_p, hidden_q, W_q, draft_tokens, uniforms, block_len)
+        if any(t.dtype != torch.bfloat16 for t in (hidden_p, W_p, hidden_q, W_q)):
+            raise TypeError("hidden states and LM-head weights must be bfloat16")
+        self.t = (hidden_p, W_p, hidden_q, W_q, draft_tokens, uniforms, block_len)
+        self.B, rows_p, self.d_p = hidden_p.shape
+        _, self.rows_q, self.d_q = hidden_q.shape
+        self.V = W_p.shape[0]
+        self.k = draft_tokens.shape[1]
+        if rows_p != self.k + 1 or W_q.shape[0] != self.V or W_p.shape[1] != self.d_p or W_q.shape[1] != self.d_q:
+            raise ValueError("shapes must be hidden_p [B,k+1,d_p], W_p [V,d_p], hidden_q [B,rows_q,d_q], W_q [V,d_q]")
+        self.temperature = float(temperature)
+        dev = hidden_p.device
+        self.workspace = _workspace(polyspec_verify_from_hidden_workspace(self.B, self.k, self.V, self.d_p, self.d_q), dev)
+        self.out = {"accepted_len": torch.empty(self.B, dtype=torch.int32, device=dev),
+                    "next_token": torch.empty(self.B, dtype=torch.int32, device=dev)}
+        self.device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.out["device_status"] = self.device_status
+        self.stream = stream
+
+    def _sizes(self):
+        return (self.B, self.k, self.V, self.d_p, self.d_q)
+
+    def launch(self):
+        hp, wp, hq, wq, tok, u, bl = self.t
+        _check(self.lib.polyspec_verify_from_hidden(
+            _ptr(hp), _ptr(wp), _ptr(hq), _ptr(wq), self.rows_q, _ptr(tok), _ptr(u), _ptr(bl), *self._sizes(), self.temperature,
+            _ptr(self.out["accepted_len"]), _ptr(self.out["next_token"]), None, None, _ptr(self.device_status),
+            _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)), "polyspec_verify_from_hidden")
+        return self.out
+
+    def project(self):
+        hp, wp, hq, wq, _, _, _ = self.t
+        _check(self.lib.polyspec_from_hidden_project(
+            _ptr(hp), _ptr(wp), _ptr(hq), _ptr(wq), self.rows_q, *self._sizes(), _ptr(self.device_status),
+            _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)), "polyspec_from_hidden_project")
+
+    def verify(self):
+        _, _, _, _, tok, u, bl = self.t
+        _check(self.lib.polyspec_from_hidden_verify(
+            self.rows_q, _ptr(tok), _ptr(u), _ptr(bl), *self._sizes(), self.temperature,
+            _ptr(self.out["accepted_len"]), _ptr(self.out["next_token"]), None, None, _ptr(self.device_status),
+            _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)), "polyspec_from_hidden_verify")
+        return self.out
 
 
 def polyspec_lm_head(hidden, W, out=None, device_status=None, stream=None):

@@ -416,32 +416,58 @@ polyspec_status polyspec_verify_from_hidden_workspace(int B, int k, int V, int d
     return POLYSPEC_OK;
 }
 
-polyspec_status polyspec_verify_from_hidden(
+namespace {
+struct FusedCall {
+    FusedLayout f;
+    float *lp, *lq;
+    char* ws;
+    cudaStream_t s;
+};
+polyspec_status fused_prepare(int rows_q, int B, int k, int V, int d_p, int d_q, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream, FusedCall* c)
+{
+    if (!workspace) return POLYSPEC_ERR_INVALID_ARG;
+    if (rows_q > k + 1) return POLYSPEC_ERR_INVALID_ARG;
+    polyspec_status st = fused_layout(B, k, rows_q, V, d_p, d_q, &c->f);
+    if (st != POLYSPEC_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return POLYSPEC_ERR_INVALID_ARG;
+    if (workspace_bytes < c->f.total) return POLYSPEC_ERR_WORKSPACE;
+    c->s = static_cast<cudaStream_t>(cuda_stream);
+    c->ws = static_cast<char*>(workspace);
+    c->lp = reinterpret_cast<float*>(c->ws + c->f.logits_p);
+    c->lq = reinterpret_cast<float*>(c->ws + c->f.logits_q);
+    return POLYSPEC_OK;
+}
+}  // namespace
+
+polyspec_status polyspec_from_hidden_project(
     const void* hidden_p, const void* W_p, const void* hidden_q, const void* W_q, int rows_q,
-    const int32_t* draft_tokens, const float* uniforms, const int32_t* block_len,
+    int B, int k, int V, int d_p, int d_q, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!hidden_p || !W_p || !hidden_q || !W_q) return POLYSPEC_ERR_INVALID_ARG;
+    if (!aligned16(hidden_p) || !aligned16(W_p) || !aligned16(hidden_q) || !aligned16(W_q)) return POLYSPEC_ERR_INVALID_ARG;
+    FusedCall c;
+    polyspec_status st = fused_prepare(rows_q, B, k, V, d_p, d_q, workspace, workspace_bytes, cuda_stream, &c);
+    if (st != POLYSPEC_OK) return st;
+    const LmHeadProblem probs[2] = {{hidden_p, W_p, B * (k + 1), d_p, c.lp}, {hidden_q, W_q, B * rows_q, d_q, c.lq}};
+    if (launch_lmhead(probs, 2, V, device_status, c.s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    return POLYSPEC_OK;
+}
+
+polyspec_status polyspec_from_hidden_verify(
+    int rows_q, const int32_t* draft_tokens, const float* uniforms, const int32_t* block_len,
     int B, int k, int V, int d_p, int d_q, float temperature,
     int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
-    if (!hidden_p || !W_p || !hidden_q || !W_q || !next_token || !accepted_len || !workspace) return POLYSPEC_ERR_INVALID_ARG;
-    if (!aligned16(hidden_p) || !aligned16(W_p) || !aligned16(hidden_q) || !aligned16(W_q)) return POLYSPEC_ERR_INVALID_ARG;
-    if (rows_q > k + 1) return POLYSPEC_ERR_INVALID_ARG;
+    if (!next_token || !accepted_len) return POLYSPEC_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || !std::isfinite(temperature)) return POLYSPEC_ERR_INVALID_ARG;
-    FusedLayout f;
-    polyspec_status st = fused_layout(B, k, rows_q, V, d_p, d_q, &f);
+    FusedCall c;
+    polyspec_status st = fused_prepare(rows_q, B, k, V, d_p, d_q, workspace, workspace_bytes, cuda_stream, &c);
     if (st != POLYSPEC_OK) return st;
-    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return POLYSPEC_ERR_INVALID_ARG;
-    if (workspace_bytes < f.total) return POLYSPEC_ERR_WORKSPACE;
-    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    char* ws = static_cast<char*>(workspace);
-    float* lp = reinterpret_cast<float*>(ws + f.logits_p);
-    float* lq = reinterpret_cast<float*>(ws + f.logits_q);
-    const LmHeadProblem probs[2] = {{hidden_p, W_p, B * (k + 1), d_p, lp}, {hidden_q, W_q, B * rows_q, d_q, lq}};
-    if (launch_lmhead(probs, 2, V, device_status, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-
     ChainArgs a;
     std::memset(&a, 0, sizeof a);
-    a.logits[0] = lp; a.logits[1] = lq;
+    a.logits[0] = c.lp; a.logits[1] = c.lq;
     a.rows[0] = k + 1; a.rows[1] = rows_q;
     a.n_models = 2;
     a.k[0] = k;
@@ -450,9 +476,27 @@ polyspec_status polyspec_verify_from_hidden(
     a.accepted_len = accepted_len; a.next_token = next_token;
     a.p_at = p_at_draft; a.q_at = q_at_draft;
     a.device_status = device_status;
-    a.workspace = ws + f.partials; a.workspace_bytes = f.total - f.partials;
-    a.stream = s;
+    a.workspace = c.ws + c.f.partials; a.workspace_bytes = c.f.total - c.f.partials;
+    a.stream = c.s;
     return run_chain(a);
+}
+
+polyspec_status polyspec_verify_from_hidden(
+    const void* hidden_p, const void* W_p, const void* hidden_q, const void* W_q, int rows_q,
+    const int32_t* draft_tokens, const float* uniforms, const int32_t* block_len,
+    int B, int k, int V, int d_p, int d_q, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    // nothing may be launched unless both halves will accept their arguments
+    if (!next_token || !accepted_len || !draft_tokens || !uniforms) return POLYSPEC_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !std::isfinite(temperature)) return POLYSPEC_ERR_INVALID_ARG;
+    polyspec_status st = polyspec_from_hidden_project(hidden_p, W_p, hidden_q, W_q, rows_q, B, k, V, d_p, d_q, device_status,
+                                                      workspace, workspace_bytes, cuda_stream);
+    if (st != POLYSPEC_OK) return st;
+    return polyspec_from_hidden_verify(rows_q, draft_tokens, uniforms, block_len, B, k, V, d_p, d_q, temperature,
+                                       accepted_len, next_token, p_at_draft, q_at_draft, device_status,
+                                       workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"
