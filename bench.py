@@ -222,6 +222,20 @@ def workload_name(args, spec):
             f"T={spec.temperature}{extra}")
 
 
+def reduce_over_ranks(times_ms, work, device, world):
+    """The multi-GPU bookkeeping: MAX over ranks of every time, SUM over ranks of every work count.
+
+    Ranks verify disjoint batches and never exchange data on the path itself; this is the only
+    collective of a run.  Returns two lists of floats (identical on every rank)."""
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), device=device, dtype=torch.float64)
+    w = torch.tensor(list(work), device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], [float(x) for x in w.tolist()]
+
+
 # ----------------------------------------------------------------------------------------- GPU arm
 def run_gpu(args, spec):
     from paper_2510_26527_b200 import binding, buildlib
@@ -306,13 +320,8 @@ def run_gpu(args, spec):
     del ws, host_models
 
     # ---- reduce over ranks: max time, summed work
-    t = torch.tensor([elapsed_ms, e2e_ms, stats_ms, walk_ms], device=dev, dtype=torch.float64)
-    w = torch.tensor([tokens_per_step, emitted_per_step], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(w, op=dist.ReduceOp.SUM)
-    elapsed_ms, e2e_ms, stats_ms, walk_ms = (float(x) for x in t.tolist())
-    tokens_all, emitted_all = (float(x) for x in w.tolist())
+    (elapsed_ms, e2e_ms, stats_ms, walk_ms), (tokens_all, emitted_all) = reduce_over_ranks(
+        [elapsed_ms, e2e_ms, stats_ms, walk_ms], [tokens_per_step, emitted_per_step], dev, world)
 
     base = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -434,13 +443,8 @@ def run_gpu_fused(args, spec):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([elapsed_ms, e2e_ms, gemm_ms, verify_ms], device=dev, dtype=torch.float64)
-    w = torch.tensor([tokens_per_step, emitted_per_step], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(w, op=dist.ReduceOp.SUM)
-    elapsed_ms, e2e_ms, gemm_ms, verify_ms = (float(x) for x in t.tolist())
-    tokens_all, emitted_all = (float(x) for x in w.tolist())
+    (elapsed_ms, e2e_ms, gemm_ms, verify_ms), (tokens_all, emitted_all) = reduce_over_ranks(
+        [elapsed_ms, e2e_ms, gemm_ms, verify_ms], [tokens_per_step, emitted_per_step], dev, world)
 
     base = None
     if rank == 0 and not args.no_cpu_baseline:

@@ -1,0 +1,64 @@
+"""The N > 1 path on CPU: two `gloo` ranks shard a workload the way `bench.py --gpus N` does.
+
+Sequences are independent, so ranks verify disjoint batches with no data-path collective; what the
+multi-rank run adds is host logic only: each rank's shard must be a distinct slice of the global
+sequence numbering (Philox counters offset by rank * B), and times / work counts are combined with
+MAX / SUM.  The verification itself runs here through the CPU oracle, since the product has no CPU path.
+"""
+import os
+import socket
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out_dir):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    from oracle import oracle as orc
+    from paper_2510_26527_b200 import synth
+    spec = synth.scaled(synth.config("cfg5", sigma=1.0), B=6, V=512)
+    d = synth.make_chain(spec, seed=3, device="cpu", batch_offset=rank * spec.B)
+    out = orc.verify_chain(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    tokens = int(out["block_len"].clip(min=0).sum())
+    emitted = int(out["out_len"][0].sum())
+    my_ms = 10.0 + 5.0 * rank
+    (t_max, t2), (tok_all, em_all) = bench.reduce_over_ranks([my_ms, 1.0], [tokens, emitted], "cpu", world)
+    np.save(os.path.join(out_dir, f"u{rank}.npy"), d["uniforms"].numpy())
+    np.save(os.path.join(out_dir, f"r{rank}.npy"), np.array([tokens, emitted, t_max, t2, tok_all, em_all]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_and_reduce(tmp_path):
+    world = 2
+    mp.spawn(_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    r = [np.load(tmp_path / f"r{i}.npy") for i in range(world)]
+    u = [np.load(tmp_path / f"u{i}.npy") for i in range(world)]
+    # the reduction: MAX of times, SUM of work, identical on both ranks
+    assert r[0][2] == r[1][2] == 15.0 and r[0][3] == r[1][3] == 1.0
+    assert r[0][4] == r[1][4] == r[0][0] + r[1][0]
+    assert r[0][5] == r[1][5] == r[0][1] + r[1][1]
+    # the shards: rank i holds sequences [i*B, (i+1)*B) of one global Philox numbering, so the shards are
+    # disjoint draws and together equal the uniforms of one batch of 2B sequences
+    sys.path.insert(0, ROOT)
+    from paper_2510_26527_b200 import synth
+    L, B, slots = u[0].shape
+    whole = synth.philox_uniforms(3, L, world * B, slots)
+    assert np.array_equal(np.concatenate(u, axis=1), whole)
+    assert not np.array_equal(u[0], u[1])
+    # every rank did real work
+    assert r[0][0] > 0 and r[1][0] > 0
