@@ -18,6 +18,15 @@ namespace {
 
 constexpr int kWalkThreads = 512;
 constexpr int kWalkWarps = kWalkThreads / 32;
+// tiles a warp loads before it computes (a float32 tile is two vectors per lane and row), and how
+// many CTAs the register budget must let an SM hold
+#ifndef POLYSPEC_WALK_UNROLL
+#define POLYSPEC_WALK_UNROLL 2
+#endif
+#ifndef POLYSPEC_WALK_CTAS_PER_SM
+#define POLYSPEC_WALK_CTAS_PER_SM 2
+#endif
+template <int DT> struct Unroll { static constexpr int value = (DT == POLYSPEC_BF16) ? POLYSPEC_WALK_UNROLL : (POLYSPEC_WALK_UNROLL + 1) / 2; };
 
 __device__ __forceinline__ float ex2f(float x)
 {
@@ -58,21 +67,55 @@ template <int DT> __device__ __forceinline__ void load8(const void* row, int v, 
     }
 }
 
+// Eight consecutive logits as loaded (one or two 16-byte vectors), unpacked later.
+template <int DT> struct RawTile;
+template <> struct RawTile<POLYSPEC_BF16> {
+    uint4 a;
+    __device__ __forceinline__ void load(const void* row, int v) { a = ld_nc(static_cast<const unsigned short*>(row) + v); }
+    __device__ __forceinline__ void unpack(float* z) const
+    {
+        z[0] = __uint_as_float(a.x << 16); z[1] = __uint_as_float(a.x & 0xffff0000u);
+        z[2] = __uint_as_float(a.y << 16); z[3] = __uint_as_float(a.y & 0xffff0000u);
+        z[4] = __uint_as_float(a.z << 16); z[5] = __uint_as_float(a.z & 0xffff0000u);
+        z[6] = __uint_as_float(a.w << 16); z[7] = __uint_as_float(a.w & 0xffff0000u);
+    }
+};
+template <> struct RawTile<POLYSPEC_F32> {
+    uint4 a, b;
+    __device__ __forceinline__ void load(const void* row, int v)
+    {
+        a = ld_nc(static_cast<const float*>(row) + v);
+        b = ld_nc(static_cast<const float*>(row) + v + 4);
+    }
+    __device__ __forceinline__ void unpack(float* z) const
+    {
+        z[0] = __uint_as_float(a.x); z[1] = __uint_as_float(a.y); z[2] = __uint_as_float(a.z); z[3] = __uint_as_float(a.w);
+        z[4] = __uint_as_float(b.x); z[5] = __uint_as_float(b.y); z[6] = __uint_as_float(b.z); z[7] = __uint_as_float(b.w);
+    }
+};
+
 struct RowStat {      // sum_v 2^(z_v * c - E) = Z
     float E;
     double Z;
 };
 
-__device__ __forceinline__ RowStat merge_partials(const float2* part, int parts)
+// One warp merges the partials of one row: lanes take partials in parallel (their loads overlap),
+// the references are maximised and the rebased sums added across the warp.  Rebasing is an exact
+// power-of-two scaling, the sum is in double.  Every lane returns the same result.
+__device__ __forceinline__ RowStat merge_partials(const float2* part, int parts, int lane)
 {
     float E = kEmptyRef;
-    for (int i = 0; i < parts; ++i) E = fmaxf(E, part[i].x);
+    for (int i = lane; i < parts; i += 32) E = fmaxf(E, part[i].x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
     double Z = 0.0;
-    for (int i = 0; i < parts; ++i) {
+    for (int i = lane; i < parts; i += 32) {
         const float2 ps = part[i];
         const float d = ps.x - E;                       // integer-valued, <= 0
         Z += (d < -1000.0f) ? static_cast<double>(ps.y) * 0.0 : ldexp(static_cast<double>(ps.y), static_cast<int>(d));
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, o);
     RowStat r;
     r.E = E;
     r.Z = Z;
@@ -142,13 +185,41 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
     const float iZq = use_q ? static_cast<float>(1.0 / sq.Z) : 0.0f;
     const float Ep = sp.E, Eq = sq.E;
 
-    for (int t = warp; t < ntiles; t += kWalkWarps) {
-        float r[8];
-        tile_resid<DT>(prow, qrow, t * kTile + lane * 8, V, c, Ep, iZp, Eq, iZq, use_q, r);
-        float x = sum8(r);
+    // kUnroll tiles per warp and step: all their loads are issued before the first is used, so a warp
+    // has kUnroll (x2 with q) 16-byte loads per lane in flight instead of one.  Each tile's sum is
+    // computed exactly as in the rescan below, whatever the grouping.
+    constexpr int kUnroll = Unroll<DT>::value;
+    for (int t0 = warp * kUnroll; t0 < ntiles; t0 += kWalkWarps * kUnroll) {
+        RawTile<DT> rp[kUnroll], rq[kUnroll];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
-        if (lane == 0) tile_sum[t] = x;
+        for (int u = 0; u < kUnroll; ++u) {
+            const int v = (t0 + u) * kTile + lane * 8;
+            if (v < V) {
+                rp[u].load(prow, v);
+                if (use_q) rq[u].load(qrow, v);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (t0 + u < ntiles) {                  // warp-uniform
+                const int v = (t0 + u) * kTile + lane * 8;
+                float r[8];
+                if (v < V) {
+                    float zp[8], zq[8];
+                    rp[u].unpack(zp);
+                    if (use_q) rq[u].unpack(zq);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) r[e] = resid(zp[e], use_q ? zq[e] : 0.0f, c, Ep, iZp, Eq, iZq, use_q);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) r[e] = 0.0f;
+                }
+                float x = sum8(r);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
+                if (lane == 0) tile_sum[t0 + u] = x;
+            }
+        }
     }
     __syncthreads();
 
@@ -228,7 +299,7 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kWalkThreads) walk_kernel(const WalkParams p)
+__global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_kernel(const WalkParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* tile_sum = reinterpret_cast<float*>(smem_raw);
@@ -271,8 +342,12 @@ __global__ void __launch_bounds__(kWalkThreads) walk_kernel(const WalkParams p)
         const char* base_q = static_cast<const char*>(p.t.logits[l + 1]) + static_cast<size_t>(b) * p.t.rows[l + 1] * row_bytes;
 
         // 1. normalisers of p rows 0..m and q rows 0..m-1
-        if (tid <= m) st_p[tid] = merge_partials(p.partials + static_cast<size_t>(grow_p + tid) * p.parts, p.parts);
-        if (tid >= 64 && tid - 64 < m) st_q[tid - 64] = merge_partials(p.partials + static_cast<size_t>(grow_q + tid - 64) * p.parts, p.parts);
+        for (int r = tid >> 5; r < 2 * m + 1; r += kWalkWarps) {          // one warp per row
+            const bool is_q = r > m;
+            const int j = is_q ? r - (m + 1) : r;
+            const RowStat st = merge_partials(p.partials + static_cast<size_t>((is_q ? grow_q : grow_p) + j) * p.parts, p.parts, tid & 31);
+            if ((tid & 31) == 0) (is_q ? st_q : st_p)[j] = st;
+        }
         __syncthreads();
 
         // 2. accept tests (warp 0; m <= 32)
