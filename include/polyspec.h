@@ -182,14 +182,16 @@ polyspec_status polyspec_verify_from_hidden(
 
 /*
  * The two halves of polyspec_verify_from_hidden, for callers that want to time or overlap them:
- *   polyspec_from_hidden_project  both LM-head projections (one launch), logits into the workspace;
+ *   polyspec_from_hidden_project  both LM-head projections (one launch): logits and, from the same
+ *                                 accumulators, every row's softmax-normaliser partials into the workspace;
  *   polyspec_from_hidden_verify   everything after it, reading the workspace the first half filled
  *                                 on the same stream.
  * Calling one after the other with the same sizes and workspace is exactly polyspec_verify_from_hidden.
  */
 polyspec_status polyspec_from_hidden_project(
     const void* hidden_p, const void* W_p, const void* hidden_q, const void* W_q, int rows_q,
-    int B, int k, int V, int d_p, int d_q, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+    int B, int k, int V, int d_p, int d_q, float temperature, int32_t* device_status, void* workspace, size_t workspace_bytes,
+    void* cuda_stream);
 polyspec_status polyspec_from_hidden_verify(
     int rows_q, const int32_t* draft_tokens, const float* uniforms, const int32_t* block_len,
     int B, int k, int V, int d_p, int d_q, float temperature,

@@ -87,7 +87,7 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_from_hidden.argtypes = [vp, vp, vp, vp, ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf,
                                                 i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
     lib.polyspec_from_hidden_project.restype = ci
-    lib.polyspec_from_hidden_project.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, i32p, vp, sz, vp]
+    lib.polyspec_from_hidden_project.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, i32p, vp, sz, vp]
     lib.polyspec_from_hidden_verify.restype = ci
     lib.polyspec_from_hidden_verify.argtypes = [ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf, i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
     lib.polyspec_lm_head.restype = ci
@@ -408,7 +408,7 @@ class FusedCall:
     def project(self):
         hp, wp, hq, wq, _, _, _ = self.t
         _check(self.lib.polyspec_from_hidden_project(
-            _ptr(hp), _ptr(wp), _ptr(hq), _ptr(wq), self.rows_q, *self._sizes(), _ptr(self.device_status),
+            _ptr(hp), _ptr(wp), _ptr(hq), _ptr(wq), self.rows_q, *self._sizes(), self.temperature, _ptr(self.device_status),
             _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)), "polyspec_from_hidden_project")
 
     def verify(self):

@@ -49,6 +49,7 @@ struct ChainArgs {
     void* workspace;
     size_t workspace_bytes;
     cudaStream_t stream;
+    int parts_override;     // > 0: the partials were written by the LM-head projection, this many per row
 };
 
 polyspec_status check_chain_shape(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt,
@@ -86,6 +87,10 @@ polyspec_status prepare_chain(const ChainArgs& a, StatsPlan* pl, StatsParams* sp
     for (int i = 0; i < a.n_models; ++i)
         if (!a.logits[i] || !aligned16(a.logits[i])) return POLYSPEC_ERR_INVALID_ARG;
     *pl = plan_stats(total_rows, a.V, a.dt);
+    if (a.parts_override > 0) {
+        pl->parts = a.parts_override;
+        pl->partial_bytes = align256(static_cast<size_t>(total_rows) * a.parts_override * sizeof(float2));
+    }
     if (a.workspace_bytes < pl->partial_bytes) return POLYSPEC_ERR_WORKSPACE;
     if (fill_rows(sp->t, a.logits, a.rows, a.n_models, a.B) < 0) return POLYSPEC_ERR_UNSUPPORTED;
     sp->V = a.V;
@@ -376,14 +381,14 @@ polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, in
     if (!hidden || !W || !logits || rows <= 0 || V <= 0 || d <= 0) return POLYSPEC_ERR_INVALID_ARG;
     if (!aligned16(hidden) || !aligned16(W) || !aligned16(logits)) return POLYSPEC_ERR_INVALID_ARG;
     if (d % 64 != 0 || static_cast<long long>(rows) * V > 0x7fffffffLL * 16) return POLYSPEC_ERR_UNSUPPORTED;
-    const LmHeadProblem pr = {hidden, W, rows, d, logits};
-    if (launch_lmhead(&pr, 1, V, device_status, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    const LmHeadProblem pr = {hidden, W, rows, d, logits, nullptr};
+    if (launch_lmhead(&pr, 1, V, 0.0f, device_status, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
 // Workspace of the fused call: fp32 logits of both models (written by the projection, read
-// back by the statistics pass and, for one row pair per sequence, by the sampling pass),
-// then the partials.
+// back for the gathers and, for one row pair per sequence, by the sampling pass), then the
+// row-statistics partials, which the projection's epilogue writes as well.
 namespace {
 struct FusedLayout { size_t logits_p, logits_q, partials, total; long long total_rows; };
 polyspec_status fused_layout(int B, int k, int rows_q, int V, int d_p, int d_q, FusedLayout* f)
@@ -398,7 +403,7 @@ polyspec_status fused_layout(int B, int k, int rows_q, int V, int d_p, int d_q, 
     size_t off = 0;
     f->logits_p = off; off += align256(static_cast<size_t>(B) * (k + 1) * V * 4);
     f->logits_q = off; off += align256(static_cast<size_t>(B) * rows_q * V * 4);
-    f->partials = off; off += align256(plan_stats(total, V, POLYSPEC_F32).partial_bytes);
+    f->partials = off; off += align256(static_cast<size_t>(total) * lmhead_parts(V) * sizeof(float2));
     f->total = off;
     f->total_rows = total;
     return POLYSPEC_OK;
@@ -442,15 +447,21 @@ polyspec_status fused_prepare(int rows_q, int B, int k, int V, int d_p, int d_q,
 
 polyspec_status polyspec_from_hidden_project(
     const void* hidden_p, const void* W_p, const void* hidden_q, const void* W_q, int rows_q,
-    int B, int k, int V, int d_p, int d_q, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+    int B, int k, int V, int d_p, int d_q, float temperature, int32_t* device_status, void* workspace, size_t workspace_bytes,
+    void* cuda_stream)
 {
     if (!hidden_p || !W_p || !hidden_q || !W_q) return POLYSPEC_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !std::isfinite(temperature)) return POLYSPEC_ERR_INVALID_ARG;
     if (!aligned16(hidden_p) || !aligned16(W_p) || !aligned16(hidden_q) || !aligned16(W_q)) return POLYSPEC_ERR_INVALID_ARG;
     FusedCall c;
     polyspec_status st = fused_prepare(rows_q, B, k, V, d_p, d_q, workspace, workspace_bytes, cuda_stream, &c);
     if (st != POLYSPEC_OK) return st;
-    const LmHeadProblem probs[2] = {{hidden_p, W_p, B * (k + 1), d_p, c.lp}, {hidden_q, W_q, B * rows_q, d_q, c.lq}};
-    if (launch_lmhead(probs, 2, V, device_status, c.s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    float2* partials = reinterpret_cast<float2*>(c.ws + c.f.partials);
+    const int parts = lmhead_parts(V);
+    const LmHeadProblem probs[2] = {{hidden_p, W_p, B * (k + 1), d_p, c.lp, partials},
+                                    {hidden_q, W_q, B * rows_q, d_q, c.lq, partials + static_cast<size_t>(B) * (k + 1) * parts}};
+    const float scale = static_cast<float>(kLog2e / static_cast<double>(temperature));
+    if (launch_lmhead(probs, 2, V, scale, device_status, c.s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
@@ -478,7 +489,9 @@ polyspec_status polyspec_from_hidden_verify(
     a.device_status = device_status;
     a.workspace = c.ws + c.f.partials; a.workspace_bytes = c.f.total - c.f.partials;
     a.stream = c.s;
-    return run_chain(a);
+    a.parts_override = lmhead_parts(V);      // the projection already left every row's partials there
+    if (!draft_tokens || !uniforms) return POLYSPEC_ERR_INVALID_ARG;
+    return run_walk(a);
 }
 
 polyspec_status polyspec_verify_from_hidden(
@@ -491,8 +504,8 @@ polyspec_status polyspec_verify_from_hidden(
     // nothing may be launched unless both halves will accept their arguments
     if (!next_token || !accepted_len || !draft_tokens || !uniforms) return POLYSPEC_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || !std::isfinite(temperature)) return POLYSPEC_ERR_INVALID_ARG;
-    polyspec_status st = polyspec_from_hidden_project(hidden_p, W_p, hidden_q, W_q, rows_q, B, k, V, d_p, d_q, device_status,
-                                                      workspace, workspace_bytes, cuda_stream);
+    polyspec_status st = polyspec_from_hidden_project(hidden_p, W_p, hidden_q, W_q, rows_q, B, k, V, d_p, d_q, temperature,
+                                                      device_status, workspace, workspace_bytes, cuda_stream);
     if (st != POLYSPEC_OK) return st;
     return polyspec_from_hidden_verify(rows_q, draft_tokens, uniforms, block_len, B, k, V, d_p, d_q, temperature,
                                        accepted_len, next_token, p_at_draft, q_at_draft, device_status,

@@ -21,11 +21,15 @@
 // Warp roles in each CTA:
 //   warp 0      TMA producer (one elected lane issues).  Both CTAs load their own tiles; all copies of a stage
 //               complete on the leader CTA's "full" barrier (no multicast anywhere)
-//   warp 6      L2 prefetch of W: 1 KiB contiguous per row, a few K blocks ahead of the TMA loads
+//   warp 10     L2 prefetch of W: 1 KiB contiguous per row, a few K blocks ahead of the TMA loads
 //   warp 1      MMA issuer (one elected lane, leader CTA only); allocates / frees TMEM in both CTAs.
 //               tcgen05.commit arrives on the "empty" / "accumulator full" barriers of both CTAs
-//   warps 2..5  epilogue: TMEM -> registers -> global, 128-byte coalesced stores per column; all
-//               eight epilogue warps of the pair arrive on the leader's "accumulator empty" barrier
+//   warps 2..9  epilogue (two warps per TMEM lane quarter, alternate 16-column chunks): TMEM ->
+//               registers -> global, 128-byte coalesced stores per column; all sixteen epilogue warps
+//               of the pair arrive on the leader's "accumulator empty" barrier.
+//               On request the epilogue also emits the row statistics of the tile (the softmax
+//               normaliser partial of each hidden row over the CTA's 128 vocabulary entries, in the
+//               format of the row-statistics kernel), so the logits need no second pass for them
 // When a column block needs at most 256 TMEM columns two accumulators alternate, so the
 // epilogue of one tile overlaps the K loop of the next.
 //
@@ -48,18 +52,22 @@ constexpr int kStagesG = 6;
 constexpr int kBytesA = kTileV * kBlockK * 2;                // 16 KiB: this CTA's rows of W
 constexpr int kBytesBMax = (kMaxCols / 2) * kBlockK * 2;     // 18 KiB: this CTA's half of the hidden tile
 constexpr int kStageBytes = kBytesA + kBytesBMax;            // 34 KiB
-constexpr int kGemmThreads = 224;
+constexpr int kEpiWarps = 8;                // warps 2..9: two per TMEM lane quarter, alternating 16-column chunks
+constexpr int kPrefetchWarp = 2 + kEpiWarps;
+constexpr int kGemmThreads = 32 * (kPrefetchWarp + 1);
 constexpr int kPrefetchK = 8;               // K blocks per L2 prefetch: 1 KiB contiguous per W row
 constexpr int kPrefetchLead = 16;           // how many K blocks the prefetch may run ahead of the TMA loads
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinLimitG = 1u << 20;
-constexpr size_t kGemmSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStagesG) * kStageBytes + 256 /* barriers */;
+constexpr int kStatStageBytes = 4 * kMaxCols * 8;            // per-quarter (E, s) of every column, merged across the four epilogue warps
+constexpr size_t kGemmSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStagesG) * kStageBytes + 256 /* barriers */ + kStatStageBytes;
 
 struct GemmJob {
     CUtensorMap map_w;      // [V, d] bf16, box {64, 128}
     CUtensorMap map_h;      // [rows, d] bf16, box {64, chunk / 2}
     const char* w;          // W itself, for the L2 prefetch that runs ahead of the TMA loads
     float* out;             // [rows, V]
+    float2* partials;       // [rows, parts] row statistics of the tile just computed, or nullptr
     int rows;
     int kblocks;            // d / 64
     int block_cols;         // columns (hidden rows) per work item, multiple of 16, <= 288
@@ -76,6 +84,8 @@ struct GemmParams {
     int vtiles;             // 256-entry vocabulary tiles
     int total_items;
     int acc_stages;         // 2 when every job's column block fits 256 TMEM columns (accumulators at columns 0 and 256), else 1
+    int parts;              // 128-entry vocabulary slices per row = 2 * vtiles (row statistics)
+    float c;                // log2(e) / T (row statistics)
     int32_t* status;
 };
 
@@ -128,6 +138,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 {
     for (uint32_t i = 0; i < kSpinLimitG; ++i) {
         if (mbar_try(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
+    }
+    return false;
+}
+
+// The same for waits that are known to be long (an epilogue warp waiting for a whole K loop): the
+// lanes sleep between polls instead of competing with the issuing warps for instruction slots.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    for (uint32_t i = 0; i < kSpinLimitG; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        __nanosleep(256);
         if ((i & 63u) == 63u && *abort_flag) return false;
     }
     return false;
@@ -198,6 +220,43 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r)
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// Largest value over the warp; NaN if any lane holds NaN.
+__device__ __forceinline__ float warp_max_nan(float x)
+{
+    float y;
+    asm volatile("redux.sync.max.NaN.f32 %0, %1, 0xffffffff;" : "=f"(y) : "f"(x));
+    return y;
+}
+// 2^d for an integer-valued d <= 0 (exact); 0 once below the normal range.
+__device__ __forceinline__ float pow2_neg(float d)
+{
+    return (d < -126.0f) ? 0.0f : __int_as_float((static_cast<int>(d) + 127) << 23);
+}
+// One butterfly step of the transposing warp reduction: a lane keeps half of its n columns, hands the
+// other half to the lane `bit` away and adds what it receives.  The references E are the same in
+// every lane, so they are only selected.
+template <int N>
+__device__ __forceinline__ void fold_columns(float* s, float* E, int lane, int bit)
+{
+    const bool upper = (lane & bit) != 0;
+#pragma unroll
+    for (int i = 0; i < N / 2; ++i) {
+        const float keep = upper ? s[i + N / 2] : s[i];
+        const float send = upper ? s[i] : s[i + N / 2];
+        s[i] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, bit));
+        E[i] = upper ? E[i + N / 2] : E[i];
+    }
+}
+__device__ __forceinline__ void mbar_arrive_local(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Work item -> (job, vocabulary tile, column block).  Items of job 0 come first; inside a job
@@ -240,12 +299,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
     const uint32_t bars = tiles + kStagesG * kStageBytes;
     const uint32_t full_bar = bars, empty_bar = full_bar + 8u * kStagesG;       // full: used in the leader only
     const uint32_t acc_full = empty_bar + 8u * kStagesG, acc_empty = acc_full + 16u;   // acc_empty: leader only
+    const uint32_t epi_bar = acc_empty + 16u;       // the four epilogue warps of this CTA meet here (bounded, unlike bar.sync)
+    float2* stat_stage = reinterpret_cast<float2*>(smem_dyn + (bars - raw) + 256);     // [4][kMaxCols]
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         loads_issued = 0;
         for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full + 8u * a, 1); mbar_init(acc_empty + 8u * a, 8); }
+        for (int a = 0; a < 2; ++a) { mbar_init(acc_full + 8u * a, 1); mbar_init(acc_empty + 8u * a, 2 * kEpiWarps); }
+        mbar_init(epi_bar, kEpiWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -301,7 +363,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             for (uint32_t i = 0; i < kSpinLimitG; ++i)
                 if (mbar_try(b, (q / kStagesG) & 1u) || *abort_p) break;
         }
-    } else if (warp == 6) {
+    } else if (warp == kPrefetchWarp) {
         // ------------------------------------------------------------------ L2 prefetch of W (both CTAs)
         // A TMA box touches 128 bytes in each of 128 rows of W that lie d * 2 bytes apart: 128 DRAM
         // pages per K block, each page visited again only a K block later.  This warp runs a little
@@ -376,10 +438,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             __syncwarp();
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
         const int quarter = warp & 3;                   // the TMEM lanes this warp may read: 32 * quarter ..
+        const int half_id = (warp - 2) >> 2;            // which of the quarter's two warps this is
         const uint32_t leader_acc_empty = cluster_addr(acc_empty, 0);
-        uint32_t tile_n = 0;
+        uint32_t tile_n = 0, epi_phase = 0;
         bool ok = true;
         for (int item = pair; ok && item < p.total_items; item += n_pairs, ++tile_n) {
             int j, vt, nb;
@@ -387,16 +450,24 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             const GemmJob& job = p.job[j];
             const int acc = tile_n % p.acc_stages;
             const uint32_t use = tile_n / p.acc_stages;
-            if (!mbar_wait(acc_full + 8u * acc, use & 1u, abort_p)) { ok = false; break; }
+            if (!mbar_wait_relaxed(acc_full + 8u * acc, use & 1u, abort_p)) { ok = false; break; }
             tc_fence_after();
             const int v = vt * kPairV + static_cast<int>(rank) * kTileV + quarter * 32 + lane;
             const int row0 = nb * job.block_cols;
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * (kTmemCols / 2);
             float* out_v = job.out + v;
-            for (int c0 = 0; c0 < job.block_cols; c0 += 16) {
+            const bool stats = job.partials != nullptr;
+            // the two warps of a quarter take alternate 16-column chunks; a warp's next chunk is already
+            // on its way from TMEM while it works on the current one
+            uint32_t nxt[16];
+            const int c_first = 16 * half_id;
+            if (c_first < job.block_cols) tmem_ld16(t_addr + c_first, nxt);
+            for (int c0 = c_first; c0 < job.block_cols; c0 += 32) {
                 uint32_t r[16];
-                tmem_ld16(t_addr + c0, r);
                 tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) r[i] = nxt[i];
+                if (c0 + 32 < job.block_cols) tmem_ld16(t_addr + c0 + 32, nxt);
                 if (v < p.V) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -404,10 +475,54 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
                         if (row < job.rows) out_v[static_cast<size_t>(row) * p.V] = __uint_as_float(r[i]);
                     }
                 }
+                if (stats) {
+                    // this warp's 32 vocabulary entries of 16 columns -> one (E, s) per column with
+                    // sum_v 2^(z_v c - E) = s, E an integer at or just above the largest z_v c
+                    float E[16], sm[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float z = (v < p.V) ? __uint_as_float(r[i]) : -INFINITY;
+                        const float m = warp_max_nan(z);
+                        E[i] = (m == -INFINITY) ? kEmptyRef : ceilf(m * p.c);
+                        sm[i] = ex2f(__fmaf_rn(z, p.c, -E[i]));
+                    }
+                    fold_columns<16>(sm, E, lane, 16);
+                    fold_columns<8>(sm, E, lane, 8);
+                    fold_columns<4>(sm, E, lane, 4);
+                    fold_columns<2>(sm, E, lane, 2);
+                    const float total = __fadd_rn(sm[0], __shfl_xor_sync(0xffffffffu, sm[0], 1));
+                    const int col = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+                    if ((lane & 1) == 0) stat_stage[quarter * kMaxCols + c0 + col] = make_float2(E[0], total);
+                }
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8u * acc);
+            if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8u * acc);     // the accumulator may be overwritten
+            if (stats) {
+                // merge the four quarters of every column and store the partial of this 128-entry slice
+                __syncwarp();
+                if (lane == 0) mbar_arrive_local(epi_bar);
+                if (!mbar_wait(epi_bar, epi_phase, abort_p)) { ok = false; break; }
+                epi_phase ^= 1u;
+                const int slice = vt * 2 + static_cast<int>(rank);
+                for (int col = (warp - 2) * 32 + lane; col < job.block_cols; col += 32 * kEpiWarps) {
+                    const int row = row0 + col;
+                    if (row < job.rows) {
+                        float2 q[4];
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) q[w] = stat_stage[w * kMaxCols + col];
+                        const float Em = fmaxf(fmaxf(q[0].x, q[1].x), fmaxf(q[2].x, q[3].x));
+                        float tot = 0.0f;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) tot = __fadd_rn(tot, __fmul_rn(q[w].y, pow2_neg(q[w].x - Em)));
+                        job.partials[static_cast<size_t>(row) * p.parts + slice] = make_float2(Em, tot);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive_local(epi_bar);
+                if (!mbar_wait(epi_bar, epi_phase, abort_p)) { ok = false; break; }     // the staging area may be reused
+                epi_phase ^= 1u;
+            }
         }
         if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
     }
@@ -461,7 +576,7 @@ bool encode_map(CUtensorMap* map, const void* base, int n_rows, int d, int box_r
 
 }  // namespace
 
-cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, int32_t* device_status, cudaStream_t stream)
+cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int32_t* device_status, cudaStream_t stream)
 {
     if (n < 1 || n > 2) return cudaErrorInvalidValue;
     cudaError_t e = get_encoder();
@@ -500,6 +615,8 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, int32_t* dev
     p.n_jobs = n;
     p.V = V;
     p.vtiles = (V + kPairV - 1) / kPairV;
+    p.parts = 2 * p.vtiles;
+    p.c = c;
     p.status = device_status;
     p.total_items = 0;
     p.acc_stages = 2;
@@ -523,6 +640,7 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, int32_t* dev
         job.rows = pr.rows;
         job.kblocks = pr.d / kBlockK;
         job.out = pr.out;
+        job.partials = pr.partials;
         job.w = static_cast<const char*>(pr.W);
         job.items = p.vtiles * job.nblocks;
         p.total_items += job.items;
