@@ -202,7 +202,8 @@ polyspec_status polyspec_from_hidden_verify(
  * polyspec_lm_head -- the projection of polyspec_verify_from_hidden on its own (the last op
  * of a model forward in Algorithm 1): logits[r, v] = sum_d hidden[r, d] * W[v, d].
  *
- *   hidden  [rows, d] bf16, W [V, d] bf16, both row-major and 16-byte aligned; d a multiple of 64
+ *   hidden  [rows, d] bf16, W [V, d] bf16, both row-major and 16-byte aligned; d a multiple of 64,
+ *           V a multiple of 4
  *   logits  out [rows, V] fp32, 16-byte aligned
  *   No workspace.  device_status as above (only POLYSPEC_ERR_TIMEOUT can be reported here).
  */

@@ -380,7 +380,7 @@ polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, in
 {
     if (!hidden || !W || !logits || rows <= 0 || V <= 0 || d <= 0) return POLYSPEC_ERR_INVALID_ARG;
     if (!aligned16(hidden) || !aligned16(W) || !aligned16(logits)) return POLYSPEC_ERR_INVALID_ARG;
-    if (d % 64 != 0 || static_cast<long long>(rows) * V > 0x7fffffffLL * 16) return POLYSPEC_ERR_UNSUPPORTED;
+    if (d % 64 != 0 || V % 4 != 0 || static_cast<long long>(rows) * V > 0x7fffffffLL * 16) return POLYSPEC_ERR_UNSUPPORTED;
     const LmHeadProblem pr = {hidden, W, rows, d, logits, nullptr};
     if (launch_lmhead(&pr, 1, V, 0.0f, device_status, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;

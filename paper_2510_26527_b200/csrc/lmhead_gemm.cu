@@ -25,10 +25,10 @@
 //   warp 1      MMA issuer (one elected lane, leader CTA only); allocates / frees TMEM in both CTAs.
 //               tcgen05.commit arrives on the "empty" / "accumulator full" barriers of both CTAs
 //   warps 2..9  epilogue (two warps per TMEM lane quarter, alternate 16-column chunks): TMEM ->
-//               registers -> global, 128-byte coalesced stores per column; all sixteen epilogue warps
-//               of the pair arrive on the leader's "accumulator empty" barrier.
+//               registers -> a 2 KiB staging tile per warp -> global by 2-D TMA store; all sixteen
+//               epilogue warps of the pair arrive on the leader's "accumulator empty" barrier.
 //               On request the epilogue also emits the row statistics of the tile (the softmax
-//               normaliser partial of each hidden row over the CTA's 128 vocabulary entries, in the
+//               normaliser partial of each hidden row over each warp's 32 vocabulary entries, in the
 //               format of the row-statistics kernel), so the logits need no second pass for them
 // When a column block needs at most 256 TMEM columns two accumulators alternate, so the
 // epilogue of one tile overlaps the K loop of the next.
@@ -59,12 +59,14 @@ constexpr int kPrefetchK = 8;               // K blocks per L2 prefetch: 1 KiB c
 constexpr int kPrefetchLead = 16;           // how many K blocks the prefetch may run ahead of the TMA loads
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinLimitG = 1u << 20;
-constexpr int kStatStageBytes = 4 * kMaxCols * 8;            // per-quarter (E, s) of every column, merged across the four epilogue warps
+constexpr int kScratchPitch = 32;                            // an epilogue warp's staging tile: [16 hidden rows][32 vocabulary entries] fp32
+constexpr int kStatStageBytes = kEpiWarps * 16 * kScratchPitch * 4;
 constexpr size_t kGemmSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStagesG) * kStageBytes + 256 /* barriers */ + kStatStageBytes;
 
 struct GemmJob {
     CUtensorMap map_w;      // [V, d] bf16, box {64, 128}
     CUtensorMap map_h;      // [rows, d] bf16, box {64, chunk / 2}
+    CUtensorMap map_out;    // [rows, V] fp32, box {32, 16}, no swizzle: the epilogue's stores
     const char* w;          // W itself, for the L2 prefetch that runs ahead of the TMA loads
     float* out;             // [rows, V]
     float2* partials;       // [rows, parts] row statistics of the tile just computed, or nullptr
@@ -84,7 +86,7 @@ struct GemmParams {
     int vtiles;             // 256-entry vocabulary tiles
     int total_items;
     int acc_stages;         // 2 when every job's column block fits 256 TMEM columns (accumulators at columns 0 and 256), else 1
-    int parts;              // 128-entry vocabulary slices per row = 2 * vtiles (row statistics)
+    int parts;              // 32-entry vocabulary slices per row = 8 * vtiles (row statistics)
     float c;                // log2(e) / T (row statistics)
     int32_t* status;
 };
@@ -164,6 +166,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+// 2-D tiled TMA store of a [16][32] fp32 staging tile; elements outside the tensor are not written.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(src) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Until the stores issued by this thread have read their shared-memory source / have completed.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // Shared-memory matrix descriptor (64 bits) of a K-major tile stored as rows of 128 bytes with
 // the 128-byte swizzle: start address >> 4 in bits 0..13, leading byte offset (unused here, 1) in
 // bits 16..29, stride byte offset 1024 >> 4 (8-row groups 1024 bytes apart) in bits 32..45,
@@ -226,36 +239,10 @@ __device__ __forceinline__ float ex2f(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// Largest value over the warp; NaN if any lane holds NaN.
-__device__ __forceinline__ float warp_max_nan(float x)
-{
-    float y;
-    asm volatile("redux.sync.max.NaN.f32 %0, %1, 0xffffffff;" : "=f"(y) : "f"(x));
-    return y;
-}
 // 2^d for an integer-valued d <= 0 (exact); 0 once below the normal range.
 __device__ __forceinline__ float pow2_neg(float d)
 {
     return (d < -126.0f) ? 0.0f : __int_as_float((static_cast<int>(d) + 127) << 23);
-}
-// One butterfly step of the transposing warp reduction: a lane keeps half of its n columns, hands the
-// other half to the lane `bit` away and adds what it receives.  The references E are the same in
-// every lane, so they are only selected.
-template <int N>
-__device__ __forceinline__ void fold_columns(float* s, float* E, int lane, int bit)
-{
-    const bool upper = (lane & bit) != 0;
-#pragma unroll
-    for (int i = 0; i < N / 2; ++i) {
-        const float keep = upper ? s[i + N / 2] : s[i];
-        const float send = upper ? s[i] : s[i + N / 2];
-        s[i] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, bit));
-        E[i] = upper ? E[i + N / 2] : E[i];
-    }
-}
-__device__ __forceinline__ void mbar_arrive_local(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -293,21 +280,26 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
     const uint32_t rank = cluster_rank();           // 0 = leader of the pair
     const uint32_t peer = rank ^ 1u;
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    // Pair i owns work items i, i + pairs, ...  Odd pairs walk their list backwards (cheap model
+    // first): neighbouring pairs are then in different phases, so the store bursts of the epilogues
+    // of some overlap the K loops of others instead of all hitting memory at once.
+    const int n_mine = (p.total_items - pair + n_pairs - 1) / n_pairs;
+    const bool backwards = (pair & 1) != 0;
+    const int first_item = backwards ? pair + (n_mine - 1) * n_pairs : pair;
+    const int item_step = backwards ? -n_pairs : n_pairs;
     // 128-byte swizzled tiles must start on a 1024-byte boundary; both CTAs use the same offsets
     const uint32_t raw = smem_addr(smem_dyn);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t bars = tiles + kStagesG * kStageBytes;
     const uint32_t full_bar = bars, empty_bar = full_bar + 8u * kStagesG;       // full: used in the leader only
     const uint32_t acc_full = empty_bar + 8u * kStagesG, acc_empty = acc_full + 16u;   // acc_empty: leader only
-    const uint32_t epi_bar = acc_empty + 16u;       // the four epilogue warps of this CTA meet here (bounded, unlike bar.sync)
-    float2* stat_stage = reinterpret_cast<float2*>(smem_dyn + (bars - raw) + 256);     // [4][kMaxCols]
+    float* stat_scratch = reinterpret_cast<float*>(smem_dyn + (bars - raw) + 256);     // per epilogue warp [16][kScratchPitch]
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         loads_issued = 0;
         for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(acc_full + 8u * a, 1); mbar_init(acc_empty + 8u * a, 2 * kEpiWarps); }
-        mbar_init(epi_bar, kEpiWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -328,7 +320,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
         uint32_t stage = 0, phase = 1;      // ring position; a fresh "empty" barrier passes a wait on parity 1
         bool ok = true;
         const uint32_t leader_full = cluster_addr(full_bar, 0);
-        for (int item = pair; ok && item < p.total_items; item += n_pairs) {
+        for (int item = first_item; ok && item >= 0 && item < p.total_items; item += item_step) {
             int j, vt, nb;
             decode_item(p, item, &j, &vt, &nb);
             const GemmJob& job = p.job[j];
@@ -371,7 +363,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
         // bursts and the TMA loads find their lines in L2.
         uint32_t it = 0;
         bool live = true;
-        for (int item = pair; live && item < p.total_items; item += n_pairs) {
+        for (int item = first_item; live && item >= 0 && item < p.total_items; item += item_step) {
             int j, vt, nb;
             decode_item(p, item, &j, &vt, &nb);
             const GemmJob& job = p.job[j];
@@ -401,7 +393,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
         if (rank == 0) {
             uint32_t stage = 0, phase = 0, tile_n = 0;
             bool ok = true;
-            for (int item = pair; ok && item < p.total_items; item += n_pairs, ++tile_n) {
+            for (int item = first_item; ok && item >= 0 && item < p.total_items; item += item_step, ++tile_n) {
                 int j, vt, nb;
                 decode_item(p, item, &j, &vt, &nb);
                 const GemmJob& job = p.job[j];
@@ -442,9 +434,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
         const int quarter = warp & 3;                   // the TMEM lanes this warp may read: 32 * quarter ..
         const int half_id = (warp - 2) >> 2;            // which of the quarter's two warps this is
         const uint32_t leader_acc_empty = cluster_addr(acc_empty, 0);
-        uint32_t tile_n = 0, epi_phase = 0;
+        float* scratch = stat_scratch + (warp - 2) * (16 * kScratchPitch);
+        uint32_t tile_n = 0;
         bool ok = true;
-        for (int item = pair; ok && item < p.total_items; item += n_pairs, ++tile_n) {
+        for (int item = first_item; ok && item >= 0 && item < p.total_items; item += item_step, ++tile_n) {
             int j, vt, nb;
             decode_item(p, item, &j, &vt, &nb);
             const GemmJob& job = p.job[j];
@@ -452,11 +445,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             const uint32_t use = tile_n / p.acc_stages;
             if (!mbar_wait_relaxed(acc_full + 8u * acc, use & 1u, abort_p)) { ok = false; break; }
             tc_fence_after();
-            const int v = vt * kPairV + static_cast<int>(rank) * kTileV + quarter * 32 + lane;
+            const int v_base = vt * kPairV + static_cast<int>(rank) * kTileV + quarter * 32;     // this warp's 32 vocabulary entries
             const int row0 = nb * job.block_cols;
             const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * (kTmemCols / 2);
-            float* out_v = job.out + v;
             const bool stats = job.partials != nullptr;
+            const int slice = (vt * 2 + static_cast<int>(rank)) * 4 + quarter;      // this warp's 32-entry slice of the row
             // the two warps of a quarter take alternate 16-column chunks; a warp's next chunk is already
             // on its way from TMEM while it works on the current one
             uint32_t nxt[16];
@@ -468,62 +461,48 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
 #pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = nxt[i];
                 if (c0 + 32 < job.block_cols) tmem_ld16(t_addr + c0 + 32, nxt);
-                if (v < p.V) {
+                if (v_base >= p.V || row0 + c0 >= job.rows) continue;      // nothing of this chunk exists (warp-uniform)
+                // registers -> staging tile [hidden row][vocabulary entry]; one TMA store writes its 16 rows of
+                // 128 bytes, the row statistics are read from the same tile
+                if (lane == 0) tma_store_wait_read();           // the previous store has read the tile
+                __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int row = row0 + c0 + i;
-                        if (row < job.rows) out_v[static_cast<size_t>(row) * p.V] = __uint_as_float(r[i]);
-                    }
-                }
+                for (int i = 0; i < 16; ++i) scratch[i * kScratchPitch + lane] = __uint_as_float(r[i]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) tma_store_2d(&job.map_out, v_base, row0 + c0, smem_addr(scratch));
                 if (stats) {
-                    // this warp's 32 vocabulary entries of 16 columns -> one (E, s) per column with
-                    // sum_v 2^(z_v c - E) = s, E an integer at or just above the largest z_v c
-                    float E[16], sm[16];
+                    // A lane owns one hidden row (col) and 16 of the 32 entries, visited in an order rotated by
+                    // col so that the lanes hit different banks; the two lanes of a row are then combined.
+                    // Result: (E, s) with sum_v 2^(z_v c - E) = s, E an integer at or just above the largest z_v c.
+                    const int col = lane & 15, e0 = (lane >> 4) * 16;
+                    float z[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float z = (v < p.V) ? __uint_as_float(r[i]) : -INFINITY;
-                        const float m = warp_max_nan(z);
-                        E[i] = (m == -INFINITY) ? kEmptyRef : ceilf(m * p.c);
-                        sm[i] = ex2f(__fmaf_rn(z, p.c, -E[i]));
+                    for (int j = 0; j < 16; ++j) {
+                        const int e = e0 + ((j + col) & 15);
+                        z[j] = (v_base + e < p.V) ? scratch[col * kScratchPitch + e] : -INFINITY;
                     }
-                    fold_columns<16>(sm, E, lane, 16);
-                    fold_columns<8>(sm, E, lane, 8);
-                    fold_columns<4>(sm, E, lane, 4);
-                    fold_columns<2>(sm, E, lane, 2);
-                    const float total = __fadd_rn(sm[0], __shfl_xor_sync(0xffffffffu, sm[0], 1));
-                    const int col = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-                    if ((lane & 1) == 0) stat_stage[quarter * kMaxCols + c0 + col] = make_float2(E[0], total);
+                    float m = z[0];
+#pragma unroll
+                    for (int j = 1; j < 16; ++j) m = fmaxf(m, z[j]);
+                    const float E = (m == -INFINITY) ? kEmptyRef : ceilf(m * p.c);
+                    float sm = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) sm = __fadd_rn(sm, ex2f(__fmaf_rn(z[j], p.c, -E)));
+                    const float E2 = __shfl_xor_sync(0xffffffffu, E, 16), s2 = __shfl_xor_sync(0xffffffffu, sm, 16);
+                    const float Em = fmaxf(E, E2);
+                    const float lo = (lane & 16) ? s2 : sm, hi = (lane & 16) ? sm : s2;       // same order in both lanes
+                    const float Elo = (lane & 16) ? E2 : E, Ehi = (lane & 16) ? E : E2;
+                    const float tot = __fadd_rn(__fmul_rn(lo, pow2_neg(Elo - Em)), __fmul_rn(hi, pow2_neg(Ehi - Em)));
+                    const int row = row0 + c0 + col;
+                    if (lane < 16 && row < job.rows) job.partials[static_cast<size_t>(row) * p.parts + slice] = make_float2(Em, tot);
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8u * acc);     // the accumulator may be overwritten
-            if (stats) {
-                // merge the four quarters of every column and store the partial of this 128-entry slice
-                __syncwarp();
-                if (lane == 0) mbar_arrive_local(epi_bar);
-                if (!mbar_wait(epi_bar, epi_phase, abort_p)) { ok = false; break; }
-                epi_phase ^= 1u;
-                const int slice = vt * 2 + static_cast<int>(rank);
-                for (int col = (warp - 2) * 32 + lane; col < job.block_cols; col += 32 * kEpiWarps) {
-                    const int row = row0 + col;
-                    if (row < job.rows) {
-                        float2 q[4];
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) q[w] = stat_stage[w * kMaxCols + col];
-                        const float Em = fmaxf(fmaxf(q[0].x, q[1].x), fmaxf(q[2].x, q[3].x));
-                        float tot = 0.0f;
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) tot = __fadd_rn(tot, __fmul_rn(q[w].y, pow2_neg(q[w].x - Em)));
-                        job.partials[static_cast<size_t>(row) * p.parts + slice] = make_float2(Em, tot);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive_local(epi_bar);
-                if (!mbar_wait(epi_bar, epi_phase, abort_p)) { ok = false; break; }     // the staging area may be reused
-                epi_phase ^= 1u;
-            }
         }
+        if (lane == 0) tma_store_wait_all();        // this thread's stores have landed before the CTA may exit
         if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
     }
 
@@ -563,6 +542,18 @@ cudaError_t get_encoder()
 
 // [n_rows, d] bf16 row-major; box = 64 elements of d (128 bytes) by box_rows rows; 128-byte swizzle;
 // rows past n_rows read as zero.
+// [n_rows, V] fp32 row-major; box = 32 vocabulary entries (128 bytes) by 16 rows, no swizzle.
+bool encode_out_map(CUtensorMap* map, float* base, int n_rows, int V)
+{
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(V), static_cast<cuuint64_t>(n_rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(V) * 4};
+    const cuuint32_t box[2] = {32, 16};
+    const cuuint32_t estr[2] = {1, 1};
+    return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool encode_map(CUtensorMap* map, const void* base, int n_rows, int d, int box_rows)
 {
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(n_rows)};
@@ -615,7 +606,7 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
     p.n_jobs = n;
     p.V = V;
     p.vtiles = (V + kPairV - 1) / kPairV;
-    p.parts = 2 * p.vtiles;
+    p.parts = 8 * p.vtiles;
     p.c = c;
     p.status = device_status;
     p.total_items = 0;
@@ -647,6 +638,7 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
         if (cols > kTmemCols / 2) p.acc_stages = 1;
         if (!encode_map(&job.map_w, pr.W, V, pr.d, kTileV)) return cudaErrorInvalidValue;
         if (!encode_map(&job.map_h, pr.hidden, pr.rows, pr.d, job.chunk / 2)) return cudaErrorInvalidValue;
+        if (!encode_out_map(&job.map_out, pr.out, pr.rows, V)) return cudaErrorInvalidValue;
     }
     const int pairs = p.total_items < g_pairs[dev] ? p.total_items : g_pairs[dev];
     lmhead_kernel<<<2 * pairs, kGemmThreads, kGemmSmemBytes, stream>>>(p);

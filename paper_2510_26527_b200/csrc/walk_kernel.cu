@@ -99,25 +99,46 @@ struct RowStat {      // sum_v 2^(z_v * c - E) = Z
     double Z;
 };
 
-// One warp merges the partials of one row: lanes take partials in parallel (their loads overlap),
-// the references are maximised and the rebased sums added across the warp.  Rebasing is an exact
-// power-of-two scaling, the sum is in double.  Every lane returns the same result.
+// Z * 2^d for an integer-valued d <= 0: an exact rescaling (0 once the gap is huge; NaN stays NaN).
+__device__ __forceinline__ double scale_pow2(double Z, float d)
+{
+    // 2^d built from its bit pattern: d is an integer in [-1000, 0] here, so the factor is a normal double
+    const double f = (d < -1000.0f) ? 0.0 : __longlong_as_double(static_cast<long long>(1023 + static_cast<int>(d)) << 52);
+    return Z * f;
+}
+
+// One warp merges the partials of one row: lanes take partials in parallel, four loads in flight
+// each, keeping a running (E, Z) that is rebased whenever a larger reference turns up; then the
+// lanes are rebased to the warp's largest reference and added.  Rebasing is an exact power-of-two
+// scaling, the sums are in double.  Every lane returns the same result.
 __device__ __forceinline__ RowStat merge_partials(const float2* part, int parts, int lane)
 {
     float E = kEmptyRef;
-    for (int i = lane; i < parts; i += 32) E = fmaxf(E, part[i].x);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) E = fmaxf(E, __shfl_xor_sync(0xffffffffu, E, o));
     double Z = 0.0;
-    for (int i = lane; i < parts; i += 32) {
-        const float2 ps = part[i];
-        const float d = ps.x - E;                       // integer-valued, <= 0
-        Z += (d < -1000.0f) ? static_cast<double>(ps.y) * 0.0 : ldexp(static_cast<double>(ps.y), static_cast<int>(d));
+    for (int i0 = lane; i0 < parts; i0 += 4 * 32) {
+        float2 ps[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + u * 32;
+            ps[u] = (i < parts) ? part[i] : make_float2(kEmptyRef, 0.0f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (ps[u].x > E) {
+                Z = scale_pow2(Z, E - ps[u].x);
+                E = ps[u].x;
+            }
+            Z += scale_pow2(static_cast<double>(ps[u].y), ps[u].x - E);
+        }
     }
+    float Ew = E;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) Ew = fmaxf(Ew, __shfl_xor_sync(0xffffffffu, Ew, o));
+    Z = scale_pow2(Z, E - Ew);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, o);
     RowStat r;
-    r.E = E;
+    r.E = Ew;
     r.Z = Z;
     return r;
 }
