@@ -30,8 +30,10 @@
 //               On request the epilogue also emits the row statistics of the tile (the softmax
 //               normaliser partial of each hidden row over each warp's 32 vocabulary entries, in the
 //               format of the row-statistics kernel), so the logits need no second pass for them
-// When a column block needs at most 256 TMEM columns two accumulators alternate, so the
-// epilogue of one tile overlaps the K loop of the next.
+// TMEM holds more than one accumulator so that the epilogue of a tile overlaps the K loop of the
+// next: two slots of 256 columns when every column block fits one, else three slots of 144 columns
+// of which a tile takes two (its two MMA chunks), so the next tile can start as soon as the first
+// of them has been drained.
 //
 // Every wait on an mbarrier is bounded.  A wait that runs out raises an abort flag in both CTAs
 // that all roles poll, sets POLYSPEC_ERR_TIMEOUT in the status word, lets copies in flight land
@@ -85,7 +87,10 @@ struct GemmParams {
     int V;
     int vtiles;             // 256-entry vocabulary tiles
     int total_items;
-    int acc_stages;         // 2 when every job's column block fits 256 TMEM columns (accumulators at columns 0 and 256), else 1
+    // TMEM is cut into n_slots accumulator slots of slot_cols columns; a tile takes slots_per_tile
+    // consecutive ones (round robin), one per MMA chunk: 2 slots of 256, 1 per tile when every column
+    // block fits 256 columns, else 3 slots of 144, 2 per tile
+    int n_slots, slots_per_tile, slot_cols;
     int parts;              // 32-entry vocabulary slices per row = 8 * vtiles (row statistics)
     float c;                // log2(e) / T (row statistics)
     int32_t* status;
@@ -292,14 +297,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t bars = tiles + kStagesG * kStageBytes;
     const uint32_t full_bar = bars, empty_bar = full_bar + 8u * kStagesG;       // full: used in the leader only
-    const uint32_t acc_full = empty_bar + 8u * kStagesG, acc_empty = acc_full + 16u;   // acc_empty: leader only
+    const uint32_t acc_full = empty_bar + 8u * kStagesG, slot_empty = acc_full + 16u;   // slot_empty[3]: leader only
     float* stat_scratch = reinterpret_cast<float*>(smem_dyn + (bars - raw) + 256);     // per epilogue warp [16][kScratchPitch]
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         loads_issued = 0;
         for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(acc_full + 8u * a, 1); mbar_init(acc_empty + 8u * a, 2 * kEpiWarps); }
+        for (int a = 0; a < 2; ++a) mbar_init(acc_full + 8u * a, 1);
+        for (int a = 0; a < 3; ++a) mbar_init(slot_empty + 8u * a, 2 * kEpiWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -397,12 +403,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
                 int j, vt, nb;
                 decode_item(p, item, &j, &vt, &nb);
                 const GemmJob& job = p.job[j];
-                const int acc = tile_n % p.acc_stages;
-                const uint32_t use = tile_n / p.acc_stages;        // how often this accumulator was used before
-                if (!mbar_wait(acc_empty + 8u * acc, (use & 1u) ^ 1u, abort_p)) { ok = false; break; }
+                // chunk i of tile t is the (slots_per_tile * t + i)-th accumulator ever used: slot = that number
+                // modulo n_slots, and the slot has been used (that number / n_slots) times before
+                const uint32_t pos0 = tile_n * p.slots_per_tile, pos1 = pos0 + p.slots_per_tile - 1;
+                const uint32_t slot0 = pos0 % p.n_slots, slot1 = pos1 % p.n_slots;
+                if (!mbar_wait(slot_empty + 8u * slot0, ((pos0 / p.n_slots) & 1u) ^ 1u, abort_p)) { ok = false; break; }
+                if (!mbar_wait(slot_empty + 8u * slot1, ((pos1 / p.n_slots) & 1u) ^ 1u, abort_p)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t idesc = instr_desc_bf16(job.chunk);
-                const uint32_t d_tmem = tmem_base + acc * (kTmemCols / 2);
+                const uint32_t d_tmem = tmem_base + slot0 * p.slot_cols, d_tmem1 = tmem_base + slot1 * p.slot_cols;
                 const uint32_t b_chunk = static_cast<uint32_t>(job.chunk >> 1) * (kBlockK * 2) >> 4;   // second MMA's B tile, in 16-byte units
                 const bool two = job.nchunks == 2;
                 for (int kb = 0; kb < job.kblocks; ++kb) {
@@ -416,14 +425,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
                             const uint32_t acc_flag = (kb | kk) != 0 ? 1u : 0u;
                             umma_bf16(d_tmem, a_lo + kk * (kMmaK * 2 >> 4), b_lo + kk * (kMmaK * 2 >> 4), idesc, acc_flag);
                             if (two)
-                                umma_bf16(d_tmem + job.chunk, a_lo + kk * (kMmaK * 2 >> 4), b_lo + b_chunk + kk * (kMmaK * 2 >> 4), idesc, acc_flag);
+                                umma_bf16(d_tmem1, a_lo + kk * (kMmaK * 2 >> 4), b_lo + b_chunk + kk * (kMmaK * 2 >> 4), idesc, acc_flag);
                         }
                         umma_commit_pair(empty_bar + 8u * stage);      // frees the stage in both CTAs once these MMAs have read it
                     }
                     __syncwarp();
                     if (++stage == kStagesG) { stage = 0; phase ^= 1u; }
                 }
-                if (ok && elect_one()) umma_commit_pair(acc_full + 8u * acc);     // accumulator complete, in both CTAs
+                if (ok && elect_one()) umma_commit_pair(acc_full + 8u * (tile_n & 1u));     // tile complete, in both CTAs
                 __syncwarp();
             }
             if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
@@ -433,7 +442,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
         // ------------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
         const int quarter = warp & 3;                   // the TMEM lanes this warp may read: 32 * quarter ..
         const int half_id = (warp - 2) >> 2;            // which of the quarter's two warps this is
-        const uint32_t leader_acc_empty = cluster_addr(acc_empty, 0);
+        const uint32_t leader_slot_empty = cluster_addr(slot_empty, 0);
         float* scratch = stat_scratch + (warp - 2) * (16 * kScratchPitch);
         uint32_t tile_n = 0;
         bool ok = true;
@@ -441,26 +450,38 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             int j, vt, nb;
             decode_item(p, item, &j, &vt, &nb);
             const GemmJob& job = p.job[j];
-            const int acc = tile_n % p.acc_stages;
-            const uint32_t use = tile_n / p.acc_stages;
-            if (!mbar_wait_relaxed(acc_full + 8u * acc, use & 1u, abort_p)) { ok = false; break; }
+            if (!mbar_wait_relaxed(acc_full + 8u * (tile_n & 1u), (tile_n >> 1) & 1u, abort_p)) { ok = false; break; }
             tc_fence_after();
+            const uint32_t pos0 = tile_n * p.slots_per_tile;
+            const uint32_t slot0 = pos0 % p.n_slots, slot1 = (pos0 + p.slots_per_tile - 1) % p.n_slots;
             const int v_base = vt * kPairV + static_cast<int>(rank) * kTileV + quarter * 32;     // this warp's 32 vocabulary entries
             const int row0 = nb * job.block_cols;
-            const uint32_t t_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * (kTmemCols / 2);
+            const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+            // TMEM address of column c of the tile: chunk 0 lives in slot0, chunk 1 (if any) in slot1
+            auto t_col = [&](int c) {
+                return c < job.chunk ? t_lane + slot0 * p.slot_cols + c : t_lane + slot1 * p.slot_cols + (c - job.chunk);
+            };
+            bool freed0 = p.slots_per_tile == 1;        // slot0 handed back already (or is the only, last one)
             const bool stats = job.partials != nullptr;
             const int slice = (vt * 2 + static_cast<int>(rank)) * 4 + quarter;      // this warp's 32-entry slice of the row
             // the two warps of a quarter take alternate 16-column chunks; a warp's next chunk is already
             // on its way from TMEM while it works on the current one
             uint32_t nxt[16];
             const int c_first = 16 * half_id;
-            if (c_first < job.block_cols) tmem_ld16(t_addr + c_first, nxt);
+            if (c_first < job.block_cols) tmem_ld16(t_col(c_first), nxt);
             for (int c0 = c_first; c0 < job.block_cols; c0 += 32) {
                 uint32_t r[16];
                 tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = nxt[i];
-                if (c0 + 32 < job.block_cols) tmem_ld16(t_addr + c0 + 32, nxt);
+                if (!freed0 && c0 >= job.chunk) {
+                    // everything this warp reads from the first slot is in registers: the next tile may overwrite it
+                    freed0 = true;
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(leader_slot_empty + 8u * slot0);
+                }
+                if (c0 + 32 < job.block_cols) tmem_ld16(t_col(c0 + 32), nxt);
                 if (v_base >= p.V || row0 + c0 >= job.rows) continue;      // nothing of this chunk exists (warp-uniform)
                 // registers -> staging tile [hidden row][vocabulary entry]; one TMA store writes its 16 rows of
                 // 128 bytes, the row statistics are read from the same tile
@@ -500,7 +521,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(leader_acc_empty + 8u * acc);     // the accumulator may be overwritten
+            if (!freed0 && lane == 0) mbar_arrive_cluster(leader_slot_empty + 8u * slot0);     // (a warp without chunks in slot1)
+            if (lane == 0) mbar_arrive_cluster(leader_slot_empty + 8u * slot1);     // the accumulator may be overwritten
         }
         if (lane == 0) tma_store_wait_all();        // this thread's stores have landed before the CTA may exit
         if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
@@ -610,7 +632,14 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
     p.c = c;
     p.status = device_status;
     p.total_items = 0;
-    p.acc_stages = 2;
+    bool wide = false;          // some column block needs more than 256 TMEM columns
+    for (int i = 0; i < n; ++i) {
+        const int c16 = (probs[i].rows + 15) / 16 * 16;
+        if (c16 > 256 && c16 <= kMaxCols) wide = true;
+    }
+    p.n_slots = wide ? 3 : 2;
+    p.slots_per_tile = wide ? 2 : 1;
+    p.slot_cols = wide ? kMaxCols / 2 : kTmemCols / 2;
     // costliest model first
     int order[2] = {0, 1};
     if (n == 2 && static_cast<long long>(probs[1].d) * probs[1].rows > static_cast<long long>(probs[0].d) * probs[0].rows) {
@@ -622,10 +651,14 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
         const LmHeadProblem& pr = probs[order[i]];
         if (pr.rows <= 0 || pr.d <= 0 || pr.d % kBlockK != 0) return cudaErrorInvalidValue;
         int cols = (pr.rows + 15) / 16 * 16;
-        if (cols > kMaxCols) cols = 256;                            // many rows: 256-column blocks, two accumulators
-        else if (cols > 256) cols = (cols + 31) / 32 * 32;          // two equal MMAs, each a multiple of 16
+        if (wide) {                                             // two MMAs per K block, each a multiple of 16 columns
+            if (cols > kMaxCols) cols = kMaxCols;
+            cols = (cols + 31) / 32 * 32;
+        } else if (cols > 256) {
+            cols = 256;                                         // many rows: 256-column blocks
+        }
         job.block_cols = cols;
-        job.nchunks = cols > 256 ? 2 : 1;
+        job.nchunks = wide ? 2 : 1;
         job.chunk = cols / job.nchunks;
         job.nblocks = (pr.rows + cols - 1) / cols;
         job.rows = pr.rows;
@@ -635,7 +668,6 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
         job.w = static_cast<const char*>(pr.W);
         job.items = p.vtiles * job.nblocks;
         p.total_items += job.items;
-        if (cols > kTmemCols / 2) p.acc_stages = 1;
         if (!encode_map(&job.map_w, pr.W, V, pr.d, kTileV)) return cudaErrorInvalidValue;
         if (!encode_map(&job.map_h, pr.hidden, pr.rows, pr.d, job.chunk / 2)) return cudaErrorInvalidValue;
         if (!encode_out_map(&job.map_out, pr.out, pr.rows, V)) return cudaErrorInvalidValue;
