@@ -67,6 +67,7 @@ struct WalkParams {
     float* p_at;                   // [B, k[0]] or nullptr (single-level call)
     float* q_at;                   // [B, k[0]] or nullptr
     int32_t* device_status;        // [1] or nullptr
+    int cluster;                   // CTAs per sequence (set by launch_walk)
 };
 
 // How the row-statistics pass is cut up for a problem size (same answer for the

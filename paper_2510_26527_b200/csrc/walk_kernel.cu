@@ -9,8 +9,11 @@
 //      max(0, P - Q) per element, per-tile sums, a scan of the tile sums, then a rescan of
 //      the one tile that contains u_s * total -> next token (inverse CDF, ascending order);
 //   4. the emitted stream (x_1..x_a, next) becomes the block of the level above.
-// Levels of one sequence depend on each other; sequences do not, so there is no
-// inter-CTA communication and no waiting of any kind.
+// Levels of one sequence depend on each other; sequences do not.  With few sequences a cluster of
+// CTAs shares one sequence: every CTA of the cluster runs the same steps on the same inputs, only the
+// row pass of step 3 is divided by tile ranges, the shares' sums and the chosen token being exchanged
+// through distributed shared memory around two cluster barriers (hardware barriers that every CTA
+// reaches unconditionally; nothing else waits).
 #include "polyspec_kernels.cuh"
 
 namespace polyspec {
@@ -189,19 +192,45 @@ __device__ __forceinline__ double warp_incl_scan(double x, int lane)
 
 struct SampleShared {
     double total;
-    double prefix;     // mass before the chosen tile
-    int tile;
+    double rank_total[8];   // mass of each CTA's share of the row (filled by the CTAs of the cluster)
     int token;
 };
+
+// A sequence may be walked by a cluster of CTAs (small batches: more SMs per sequence).  Every CTA
+// runs the same control flow on the same inputs; only the row pass is divided, by tile ranges.
+struct ClusterCtx {
+    int size;       // CTAs per sequence: 1, 2, 4 or 8
+    int rank;
+};
+
+__device__ __forceinline__ uint32_t peer_addr(const void* local, int rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(local))), "r"(rank));
+    return r;
+}
+// All threads of all CTAs of the cluster; also orders their shared-memory traffic (release / acquire).
+__device__ __forceinline__ void cluster_barrier(const ClusterCtx& cl)
+{
+    if (cl.size > 1) {
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    } else {
+        __syncthreads();
+    }
+}
 
 // Inverse CDF of the residual (use_q) or of P (bonus / fallback) at uniform u.
 // Returns the token (same value in every thread) and the total mass through *total_out.
 template <int DT>
 __device__ int sample_row(const void* prow, const void* qrow, int V, float c, RowStat sp, RowStat sq, bool use_q,
-                          float u, float* tile_sum, SampleShared* sh, double* total_out)
+                          float u, float* tile_sum, SampleShared* sh, double* total_out, const ClusterCtx cl)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ntiles = (V + kTile - 1) / kTile;
+    // this CTA's share of the row: tiles [tlo, thi)
+    const int tiles_per_rank = (ntiles + cl.size - 1) / cl.size;
+    const int tlo = min(cl.rank * tiles_per_rank, ntiles), thi = min(tlo + tiles_per_rank, ntiles);
     const float iZp = static_cast<float>(1.0 / sp.Z);
     const float iZq = use_q ? static_cast<float>(1.0 / sq.Z) : 0.0f;
     const float Ep = sp.E, Eq = sq.E;
@@ -210,7 +239,7 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
     // has kUnroll (x2 with q) 16-byte loads per lane in flight instead of one.  Each tile's sum is
     // computed exactly as in the rescan below, whatever the grouping.
     constexpr int kUnroll = Unroll<DT>::value;
-    for (int t0 = warp * kUnroll; t0 < ntiles; t0 += kWalkWarps * kUnroll) {
+    for (int t0 = tlo + warp * kUnroll; t0 < thi; t0 += kWalkWarps * kUnroll) {
         RawTile<DT> rp[kUnroll], rq[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
@@ -222,7 +251,7 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
         }
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            if (t0 + u < ntiles) {                  // warp-uniform
+            if (t0 + u < thi) {                     // warp-uniform
                 const int v = (t0 + u) * kTile + lane * 8;
                 float r[8];
                 if (v < V) {
@@ -244,75 +273,103 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
     }
     __syncthreads();
 
+    // each lane of warp 0 owns a contiguous run of the CTA's tiles; tile sums are added in double, in order
+    const int nt = thi - tlo, per = (nt + 31) / 32;
+    const int t0 = tlo + min(lane * per, nt), t1 = min(t0 + per, thi);
+    double mine = 0.0, incl = 0.0;
     if (warp == 0) {
-        // each lane owns a contiguous run of tiles; tile sums are added in double, in order
-        const int per = (ntiles + 31) / 32;
-        const int t0 = min(lane * per, ntiles), t1 = min(t0 + per, ntiles);
-        double mine = 0.0;
         for (int t = t0; t < t1; ++t) mine += static_cast<double>(tile_sum[t]);
-        const double incl = warp_incl_scan(mine, lane);
-        const double total = __shfl_sync(0xffffffffu, incl, 31);
-        const double target = static_cast<double>(u) * total;
-        const unsigned hit = __ballot_sync(0xffffffffu, incl > target);
-        const unsigned has_mass = __ballot_sync(0xffffffffu, mine > 0.0);
-        // the first lane whose running sum passes the target; if the uniform was not below 1
-        // or rounding leaves none, the last lane that holds any mass
-        const int owner = hit ? (__ffs(hit) - 1) : (has_mass ? (31 - __clz(has_mass)) : -1);
-        int tile = -1;
-        double prefix = 0.0;
-        if (owner >= 0) {
-            if (lane == owner) {
-                double run = incl - mine;
-                for (int t = t0; t < t1; ++t) {
-                    const double nxt = run + static_cast<double>(tile_sum[t]);
-                    if (nxt > target) { tile = t; prefix = run; break; }
-                    run = nxt;
-                }
-                if (tile < 0) {                       // take the lane's last non-empty tile
-                    run = incl - mine;
-                    for (int t = t0; t < t1; ++t) {
-                        if (tile_sum[t] > 0.0f) { tile = t; prefix = run; }
-                        run += static_cast<double>(tile_sum[t]);
-                    }
-                }
-            }
-            tile = __shfl_sync(0xffffffffu, tile, owner);
-            prefix = __shfl_sync(0xffffffffu, prefix, owner);
-        }
-        int token = -1;
-        if (tile >= 0) {
-            float r[8];
-            tile_resid<DT>(prow, qrow, tile * kTile + lane * 8, V, c, Ep, iZp, Eq, iZq, use_q, r);
-            double lane_sum = 0.0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) lane_sum += static_cast<double>(r[e]);
-            const double lincl = warp_incl_scan(lane_sum, lane);
-            const double tt = target - prefix;
-            const unsigned lhit = __ballot_sync(0xffffffffu, lincl > tt);
-            const unsigned lpos = __ballot_sync(0xffffffffu, lane_sum > 0.0);
-            // the first lane whose running sum passes the target; if rounding leaves none, the last lane with mass
-            const int pick = lhit ? (__ffs(lhit) - 1) : (lpos ? (31 - __clz(lpos)) : -1);
-            if (pick >= 0 && lane == pick) {
-                double run = lincl - lane_sum;
-                int last_pos = -1;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    if (token < 0) {
-                        run += static_cast<double>(r[e]);
-                        if (r[e] > 0.0f) last_pos = e;
-                        if (run > tt) token = tile * kTile + lane * 8 + e;
-                    }
-                }
-                if (token < 0 && last_pos >= 0) token = tile * kTile + lane * 8 + last_pos;
-            }
-            if (pick >= 0) token = __shfl_sync(0xffffffffu, token, pick);
-        }
-        if (lane == 0) {
-            sh->total = total;
-            sh->token = token;
+        incl = warp_incl_scan(mine, lane);
+        const double share = __shfl_sync(0xffffffffu, incl, 31);
+        if (cl.size == 1) {
+            if (lane == 0) sh->rank_total[0] = share;
+        } else if (lane < cl.size) {            // lane r tells CTA r this CTA's share
+            asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(peer_addr(&sh->rank_total[cl.rank], lane)), "d"(share) : "memory");
         }
     }
-    __syncthreads();
+    cluster_barrier(cl);
+
+    if (warp == 0) {
+        // total mass and the CTA whose share contains u * total (the same arithmetic in every CTA)
+        double total = 0.0;
+        for (int r = 0; r < cl.size; ++r) total += sh->rank_total[r];
+        const double target = static_cast<double>(u) * total;
+        int owner_rank = -1, last_mass = -1;
+        double base = 0.0, last_base = 0.0, cum = 0.0;
+        for (int r = 0; r < cl.size; ++r) {
+            const double nxt = cum + sh->rank_total[r];
+            if (owner_rank < 0 && nxt > target) { owner_rank = r; base = cum; }
+            if (sh->rank_total[r] > 0.0) { last_mass = r; last_base = cum; }
+            cum = nxt;
+        }
+        if (owner_rank < 0) { owner_rank = last_mass; base = last_base; }      // u not below 1, or rounding
+        int token = -1;
+        if (owner_rank == cl.rank) {
+            const unsigned hit = __ballot_sync(0xffffffffu, base + incl > target);
+            const unsigned has_mass = __ballot_sync(0xffffffffu, mine > 0.0);
+            // the first lane whose running sum passes the target; if rounding leaves none, the last lane
+            // that holds any mass
+            const int owner = hit ? (__ffs(hit) - 1) : (has_mass ? (31 - __clz(has_mass)) : -1);
+            int tile = -1;
+            double prefix = 0.0;
+            if (owner >= 0) {
+                if (lane == owner) {
+                    double run = base + (incl - mine);
+                    for (int t = t0; t < t1; ++t) {
+                        const double nxt = run + static_cast<double>(tile_sum[t]);
+                        if (nxt > target) { tile = t; prefix = run; break; }
+                        run = nxt;
+                    }
+                    if (tile < 0) {                       // take the lane's last non-empty tile
+                        run = base + (incl - mine);
+                        for (int t = t0; t < t1; ++t) {
+                            if (tile_sum[t] > 0.0f) { tile = t; prefix = run; }
+                            run += static_cast<double>(tile_sum[t]);
+                        }
+                    }
+                }
+                tile = __shfl_sync(0xffffffffu, tile, owner);
+                prefix = __shfl_sync(0xffffffffu, prefix, owner);
+            }
+            if (tile >= 0) {
+                float r[8];
+                tile_resid<DT>(prow, qrow, tile * kTile + lane * 8, V, c, Ep, iZp, Eq, iZq, use_q, r);
+                double lane_sum = 0.0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) lane_sum += static_cast<double>(r[e]);
+                const double lincl = warp_incl_scan(lane_sum, lane);
+                const double tt = target - prefix;
+                const unsigned lhit = __ballot_sync(0xffffffffu, lincl > tt);
+                const unsigned lpos = __ballot_sync(0xffffffffu, lane_sum > 0.0);
+                // the first lane whose running sum passes the target; if rounding leaves none, the last lane with mass
+                const int pick = lhit ? (__ffs(lhit) - 1) : (lpos ? (31 - __clz(lpos)) : -1);
+                if (pick >= 0 && lane == pick) {
+                    double run = lincl - lane_sum;
+                    int last_pos = -1;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if (token < 0) {
+                            run += static_cast<double>(r[e]);
+                            if (r[e] > 0.0f) last_pos = e;
+                            if (run > tt) token = tile * kTile + lane * 8 + e;
+                        }
+                    }
+                    if (token < 0 && last_pos >= 0) token = tile * kTile + lane * 8 + last_pos;
+                }
+                if (pick >= 0) token = __shfl_sync(0xffffffffu, token, pick);
+            }
+        }
+        if (lane == 0) sh->total = total;
+        // the CTA that holds the token tells every CTA (with no mass anywhere, CTA 0 reports -1)
+        if (cl.rank == (owner_rank < 0 ? 0 : owner_rank)) {
+            if (cl.size == 1) {
+                if (lane == 0) sh->token = token;
+            } else if (lane < cl.size) {
+                asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_addr(&sh->token, lane)), "r"(token) : "memory");
+            }
+        }
+    }
+    cluster_barrier(cl);
     *total_out = sh->total;
     const int token = sh->token;
     __syncthreads();          // sh and tile_sum are reused by the next pass
@@ -332,7 +389,12 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
     __shared__ SampleShared sh_sample;
 
     constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
-    const int b = blockIdx.x;
+    // blockIdx.x = sequence * cluster size + rank in the cluster; only rank 0 writes results
+    ClusterCtx cl;
+    cl.size = p.cluster;
+    cl.rank = static_cast<int>(blockIdx.x) % p.cluster;
+    const bool writer = cl.rank == 0;
+    const int b = static_cast<int>(blockIdx.x) / p.cluster;
     const int tid = threadIdx.x;
     const int L = p.n_levels;
     const size_t row_bytes = static_cast<size_t>(p.V) * ELEM;
@@ -348,12 +410,12 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
         const int kl = p.k[l];
         const size_t lb = static_cast<size_t>(l) * p.B + b;
         if (dead) {               // an unusable input below: this level reports -1 as well
-            if (tid == 0) {
+            if (writer && tid == 0) {
                 p.accepted_len[lb] = -1;
                 if (p.block_len) p.block_len[lb] = -1;
                 if (p.out_len) p.out_len[lb] = -1;
             }
-            if (p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
+            if (writer && p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
             continue;
         }
         const int m = min(kl, stream_len);
@@ -391,8 +453,8 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
                     qf = static_cast<float>(Q);
                 }
             }
-            if (l == 0 && p.p_at && tid < kl) p.p_at[static_cast<size_t>(b) * kl + tid] = pf;
-            if (l == 0 && p.q_at && tid < kl) p.q_at[static_cast<size_t>(b) * kl + tid] = qf;
+            if (writer && l == 0 && p.p_at && tid < kl) p.p_at[static_cast<size_t>(b) * kl + tid] = pf;
+            if (writer && l == 0 && p.q_at && tid < kl) p.q_at[static_cast<size_t>(b) * kl + tid] = qf;
             const unsigned rej_mask = __ballot_sync(0xffffffffu, rej);
             const unsigned bad_mask = __ballot_sync(0xffffffffu, bad);
             const int first_rej = rej_mask ? (__ffs(rej_mask) - 1) : m;
@@ -408,14 +470,14 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
         const int a = sh_a;
         if (sh_bad) {
             dead = true;
-            if (tid == 0) {
+            if (writer && tid == 0) {
                 p.accepted_len[lb] = -1;
                 if (p.block_len) p.block_len[lb] = -1;
                 if (p.out_len) p.out_len[lb] = -1;
                 if (p.next_token) p.next_token[b] = -1;
                 if (p.device_status) atomicCAS(p.device_status, 0, static_cast<int>(POLYSPEC_ERR_BAD_INPUT_ON_DEVICE));
             }
-            if (p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
+            if (writer && p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
             __syncthreads();
             continue;
         }
@@ -428,19 +490,19 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
         const RowStat sp = st_p[a];
         const RowStat sq = use_q ? st_q[a] : sp;
         double total = 0.0;
-        int next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, use_q, u_s, tile_sum, &sh_sample, &total);
+        int next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, use_q, u_s, tile_sum, &sh_sample, &total, cl);
         if (use_q && !(total > 0.0)) {          // residual vanished in floating point: sample P instead
-            next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, false, u_s, tile_sum, &sh_sample, &total);
+            next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, false, u_s, tile_sum, &sh_sample, &total, cl);
         }
 
         // 4. outputs and hand-off
-        if (tid == 0) {
+        if (writer && tid == 0) {
             p.accepted_len[lb] = a;
             if (p.block_len) p.block_len[lb] = m;
             if (p.out_len) p.out_len[lb] = a + 1;
             if (p.next_token) p.next_token[b] = next;
         }
-        if (p.out_tokens && tid <= p.kmax)
+        if (writer && p.out_tokens && tid <= p.kmax)
             p.out_tokens[lb * (p.kmax + 1) + tid] = (tid < a) ? tok[tid] : (tid == a ? next : -1);
         __syncthreads();
         if (tid == 0) tok[a] = next;
@@ -451,16 +513,45 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
 
 }  // namespace
 
-cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p, cudaStream_t stream)
+namespace {
+int g_walk_sms[64] = {0};
+}
+
+cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p_in, cudaStream_t stream)
 {
-    if (p.B <= 0) return cudaSuccess;
-    const int ntiles = (p.V + kTile - 1) / kTile;
+    if (p_in.B <= 0) return cudaSuccess;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (g_walk_sms[dev] == 0) {
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        g_walk_sms[dev] = sms > 0 ? sms : 148;
+    }
+    const int ntiles = (p_in.V + kTile - 1) / kTile;
+    // Few sequences: a cluster of up to 8 CTAs walks each one, so that the row passes use more SMs.
+    // The largest power of two that still lets every CTA be resident at once (two per SM).
+    WalkParams p = p_in;
+    p.cluster = 1;
+    while (p.cluster < 8 && static_cast<long long>(p.B) * (2 * p.cluster) <= 2LL * g_walk_sms[dev] && 2 * p.cluster <= ntiles)
+        p.cluster *= 2;
     const size_t smem = static_cast<size_t>(ntiles) * sizeof(float);
-    if (dt == POLYSPEC_BF16)
-        walk_kernel<POLYSPEC_BF16><<<p.B, kWalkThreads, smem, stream>>>(p);
-    else
-        walk_kernel<POLYSPEC_F32><<<p.B, kWalkThreads, smem, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(p.B) * p.cluster);
+    cfg.blockDim = dim3(kWalkThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = static_cast<unsigned>(p.cluster);
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (dt == POLYSPEC_BF16) return cudaLaunchKernelEx(&cfg, walk_kernel<POLYSPEC_BF16>, p);
+    return cudaLaunchKernelEx(&cfg, walk_kernel<POLYSPEC_F32>, p);
 }
 
 }  // namespace polyspec
