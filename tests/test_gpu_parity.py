@@ -245,3 +245,70 @@ def test_chain_host_entry_point_matches_device_entry_point():
     for key in ("accepted_len", "block_len", "out_tokens", "out_len"):
         assert (out[key].numpy() == ref[key]).all()
     assert out["host_status"][0] == 0
+
+
+# ------------------------------------------------------------------ limits of the interface
+def test_level_with_the_largest_block(oracle):
+    """k = POLYSPEC_MAX_K: a close drafter, so long accepted prefixes occur, up to the whole block."""
+    B, k, V = 40, binding.MAX_K, 768
+    spec = synth.ChainSpec("maxk", 2, B, V, torch.float32, (k,), 1.0, 3.0, (0.15,), False)
+    d = synth.make_chain(spec, seed=11, device=DEV)
+    lp, lq = d["models"]
+    out = _np(binding.polyspec_verify_level(lp, lq, d["draft_tokens"], d["uniforms"][0], 1.0, want_probs=True))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), d["draft_tokens"].cpu(), d["uniforms"][0].cpu(), 1.0, threads=8)
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B * (k + 1), "k = 32")
+    assert ora["accepted_len"].max() >= 16 and ora["accepted_len"].min() < ora["accepted_len"].max()
+
+
+def test_chain_with_the_largest_number_of_models(oracle):
+    n = binding.MAX_MODELS
+    spec = synth.ChainSpec("max_models", n, 20, 512, torch.bfloat16, (3,) * (n - 1), 0.8, 3.0, (0.4,) * (n - 1), True)
+    d = synth.make_chain(spec, seed=12, device=DEV)
+    out = _run_chain(d)
+    ora = _oracle_chain(oracle, d)
+    counts, bad = H.compare_chain(out, ora)
+    _assert_parity(counts, bad, 20 * 3 * (n - 1), "8 models")
+    assert out["device_status"][0] == 0
+
+
+def test_level_with_the_largest_vocabulary(oracle):
+    """V = 8192 tiles of 256: the most the sampling pass keeps tile sums for; one more tile is refused."""
+    V, B, k = 8192 * 256, 2, 1
+    spec = synth.ChainSpec("maxv", 2, B, V, torch.bfloat16, (k,), 1.0, 3.0, (1.0,), False)
+    d = synth.make_chain(spec, seed=13, device=DEV)
+    lp, lq = d["models"]
+    out = _np(binding.polyspec_verify_level(lp, lq, d["draft_tokens"], d["uniforms"][0], 1.0))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), d["draft_tokens"].cpu(), d["uniforms"][0].cpu(), 1.0, threads=2)
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B * 2, "V = 2 Mi")
+    with pytest.raises(binding.PolyspecError) as err:
+        binding.polyspec_verify_level_workspace(B, k, V + 256, binding.BF16)
+    assert err.value.status == binding.ERR_UNSUPPORTED
+
+
+def test_chain_with_empty_blocks_samples_the_bonus_row(oracle):
+    """block_len = 0: nothing to test, the token is drawn from row 0 of p (the bonus row of an empty block)."""
+    B, k, V = 9, 3, 2048
+    g = torch.Generator(device=DEV).manual_seed(14)
+    lp = torch.randn((B, k + 1, V), generator=g, device=DEV) * 3
+    lq = torch.randn((B, k, V), generator=g, device=DEV) * 3
+    tok = torch.randint(0, V, (B, k), generator=g, device=DEV, dtype=torch.int32)
+    u = torch.from_numpy(synth.philox_uniforms(14, 1, B, k + 1)[0]).to(DEV)
+    bl = torch.zeros(B, dtype=torch.int32, device=DEV)
+    out = _np(binding.polyspec_verify_level(lp, lq, tok, u, 1.0, block_len=bl))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), 1.0, block_len=bl.cpu())
+    assert (out["accepted_len"] == 0).all()
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B, "block_len = 0")
+
+
+@pytest.mark.parametrize("B", [1, 2, 37, 75, 149, 300])
+def test_chain_batch_sizes_across_the_cluster_thresholds(oracle, B):
+    """The walk uses 8, 4, 2 or 1 CTAs per sequence depending on the batch; the results must not depend on it."""
+    spec = synth.scaled(synth.config("cfg3"), B=B, V=6144 + 8)
+    d = synth.make_chain(spec, seed=15 + B, device=DEV)
+    out = _run_chain(d)
+    ora = _oracle_chain(oracle, d)
+    counts, bad = H.compare_chain(out, ora)
+    _assert_parity(counts, bad, B * sum(spec.k), f"cfg3 recipe at B={B}")
