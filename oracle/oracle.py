@@ -52,6 +52,9 @@ def _load():
         lib.pso_verify_chain_seq.argtypes = [ctypes.POINTER(vp), i32p, ctypes.c_int, i32p, i32p, ctypes.c_int,
                                              f32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int,
                                              ctypes.c_double, i32p, i32p, i32p, i32p, f64p, f64p, i32p, f64p]
+        lib.pso_verify_chain_greedy_seq.restype = ctypes.c_int
+        lib.pso_verify_chain_greedy_seq.argtypes = [ctypes.POINTER(vp), i32p, ctypes.c_int, i32p, i32p, ctypes.c_int, ctypes.c_int,
+                                                    ctypes.c_int64, ctypes.c_int, i32p, i32p, i32p, i32p]
         _lib = lib
     return _lib
 
@@ -216,6 +219,45 @@ def verify_chain(models, k, draft_tokens, uniforms, temperature, bottom_len=None
         out["accepted_len"][:, b] = acc; out["block_len"][:, b] = blk; out["out_len"][:, b] = olen
         out["out_tokens"][:, b, :] = otok; out["accept_margin"][:, b, :] = marg
         out["sample_info"][:, b, :] = sinfo; out["fallback"][:, b] = fb; out["status"][b] = st
+
+    _run(one, list(range(B)) if seqs is None else list(seqs), threads)
+    del bufs
+    return out
+
+
+def verify_chain_greedy(models, k, draft_tokens, bottom_len=None, threads=1, seqs=None):
+    """The chain under greedy matching (Sections 3.1 and 4.5): a token is accepted iff it is the
+    verifier's arg max, the emitted token is the verifier's arg max after the accepted prefix.
+
+    models as in verify_chain; the last one (the drafter's logits) is not read and may be None.
+    Returns accepted_len, block_len, out_len [n-1, B], out_tokens [n-1, B, kmax+1], status [B].
+    """
+    lib = _load()
+    n = len(models)
+    L = n - 1
+    bufs = [_buf(m) if m is not None else None for m in models]
+    code = bufs[0][1]
+    B, _, V = bufs[0][2]
+    k = np.ascontiguousarray(k, dtype=np.int32)
+    kmax = int(k.max())
+    tok = _i32(draft_tokens)
+    assert tok.shape == (B, int(k[-1]))
+    nrows = np.array([b[2][1] if b is not None else int(k[-1]) for b in bufs], dtype=np.int32)
+    bl = np.full(B, int(k[-1]), np.int32) if bottom_len is None else _i32(bottom_len)
+    out = {"accepted_len": np.full((L, B), -1, np.int32), "block_len": np.full((L, B), -1, np.int32),
+           "out_tokens": np.full((L, B, kmax + 1), -1, np.int32), "out_len": np.full((L, B), -1, np.int32),
+           "status": np.zeros(B, np.int32)}
+
+    def one(b):
+        ptrs = (ctypes.c_void_p * n)(*[(bufs[i][0] + b * int(nrows[i]) * V * bufs[i][3]) if bufs[i] is not None else None
+                                       for i in range(n)])
+        acc = np.empty(L, np.int32); blk = np.empty(L, np.int32); olen = np.empty(L, np.int32)
+        otok = np.empty((L, kmax + 1), np.int32)
+        st = lib.pso_verify_chain_greedy_seq(ptrs, _p(nrows, ctypes.c_int32), n, _p(k, ctypes.c_int32), _p(tok[b], ctypes.c_int32),
+                                             int(bl[b]), kmax, V, code, _p(acc, ctypes.c_int32), _p(blk, ctypes.c_int32),
+                                             _p(otok, ctypes.c_int32), _p(olen, ctypes.c_int32))
+        out["accepted_len"][:, b] = acc; out["block_len"][:, b] = blk; out["out_len"][:, b] = olen
+        out["out_tokens"][:, b, :] = otok; out["status"][b] = st
 
     _run(one, list(range(B)) if seqs is None else list(seqs), threads)
     del bufs

@@ -287,3 +287,81 @@ int pso_verify_chain_seq(const void* const* model_rows, const int32_t* model_nro
     free(stream);
     return status;
 }
+
+/*
+ * Greedy matching, the other verification rule Section 3.1 names ("speculative sampling,
+ * greedy matching, or another verification rule") and the one Section 4.5 compares
+ * acceptance-length variance against: a block token is accepted iff it is the verifier's
+ * most likely token at its position, the loop breaks at the first mismatch, and the
+ * token emitted after the accepted prefix is the verifier's most likely token there (at
+ * the first mismatch, or in the bonus row after a fully accepted block).  No uniforms, no
+ * temperature (the arg max does not depend on it) and no drafter distribution: only the
+ * verifier's rows and the block tokens matter.
+ *
+ * Arg max of one row: the first index holding the largest logit.  A row holding NaN or
+ * +inf, or no finite logit, is unusable, as in the sampling rule.
+ */
+int pso_argmax_row(const void* row, int dtype, int64_t V, int32_t* arg)
+{
+    if (!row || !arg || V <= 0) return PSO_BAD_ARG;
+    double best = -INFINITY;
+    int64_t at = -1;
+    for (int64_t v = 0; v < V; ++v) {
+        double z = pso_load(row, dtype, v);
+        if (isnan(z) || (isinf(z) && z > 0)) return PSO_BAD_ROW_NAN;
+        if (z > best) { best = z; at = v; }
+    }
+    if (at < 0) return PSO_BAD_ROW_EMPTY;
+    *arg = (int32_t)at;
+    return PSO_OK;
+}
+
+/*
+ * The chain under greedy matching, one sequence; arguments as in pso_verify_chain_seq
+ * without uniforms and temperature.  model_rows[n-1] (the bottom drafter's logits) is
+ * never read and may be NULL.
+ */
+int pso_verify_chain_greedy_seq(const void* const* model_rows, const int32_t* model_nrows, int n,
+                                const int32_t* k, const int32_t* draft_tokens, int bottom_len, int kmax,
+                                int64_t V, int dtype,
+                                int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len)
+{
+    if (n < 2 || !model_rows || !model_nrows || !k || kmax < 1) return PSO_BAD_ARG;
+    int L = n - 1;
+    for (int l = 0; l < L; ++l) {
+        accepted_len[l] = -1; block_len[l] = -1; out_len[l] = -1;
+        for (int j = 0; j <= kmax; ++j) out_tokens[(size_t)l * (kmax + 1) + j] = -1;
+        if (k[l] < 0 || k[l] > kmax || model_nrows[l] < k[l] + 1 || !model_rows[l]) return PSO_BAD_ARG;
+    }
+    if (bottom_len < 0 || bottom_len > k[L - 1]) return PSO_BAD_ARG;
+    int32_t* stream = (int32_t*)malloc(sizeof(int32_t) * (size_t)(kmax + 2));
+    if (!stream) return PSO_BAD_ARG;
+    int stream_len = bottom_len;
+    for (int j = 0; j < bottom_len; ++j) stream[j] = draft_tokens[j];
+    int status = PSO_OK;
+    for (int l = L - 1; l >= 0 && status == PSO_OK; --l) {
+        int m = stream_len < k[l] ? stream_len : k[l];
+        int a = 0;
+        int32_t next = -1;
+        for (int j = 0; j <= m; ++j) {          /* row j scores position j; row m is the bonus row */
+            if (j < m && (stream[j] < 0 || (int64_t)stream[j] >= V)) { status = PSO_BAD_TOKEN; break; }
+            int32_t top;
+            status = pso_argmax_row(pso_row(model_rows[l], dtype, V, j), dtype, V, &top);
+            if (status) break;
+            if (j < m && stream[j] == top) { a += 1; continue; }
+            next = top;                          /* first mismatch, or the bonus row */
+            break;
+        }
+        if (status) break;
+        accepted_len[l] = a;
+        block_len[l] = m;
+        out_len[l] = a + 1;
+        int32_t* out = out_tokens + (size_t)l * (kmax + 1);
+        for (int j = 0; j < a; ++j) out[j] = stream[j];
+        out[a] = next;
+        stream[a] = next;
+        stream_len = a + 1;
+    }
+    free(stream);
+    return status;
+}
