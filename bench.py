@@ -486,6 +486,61 @@ def run_gpu_fused(args, spec):
         dist.destroy_process_group()
 
 
+def run_gpu_greedy(args, spec):
+    """--rule greedy: the chain under greedy matching (one arg-max pass over the verifiers' logits + a small walk)."""
+    from paper_2510_26527_b200 import binding, buildlib
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: libpolyspec has no CPU path")
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise RuntimeError("--rule greedy is a single-GPU measurement")
+    dev = torch.device("cuda", 0)
+    buildlib.build()
+    binding.load_library()
+    data = synth.make_chain(spec, seed=args.seed, device=dev)
+    kb = data["k"][-1]
+    g = torch.Generator(device=dev).manual_seed(args.seed + 1)
+    top = data["models"][-2][:, :kb].float().argmax(-1)
+    flip = torch.rand(top.shape, generator=g, device=dev) < 0.1
+    draft = torch.where(flip, torch.randint(0, spec.V, top.shape, generator=g, device=dev), top).to(torch.int32).contiguous()
+    verifiers = data["models"][:-1]
+    rows = [int(m.shape[1]) for m in verifiers] + [kb]
+    ws = torch.empty(max(256, binding.polyspec_verify_chain_greedy_workspace(data["k"], rows, spec.B, spec.V, binding._dt(verifiers[0]))),
+                     dtype=torch.uint8, device=dev)
+    out = binding.chain_outputs(spec.n_models - 1, spec.B, spec.kmax, dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    call = lambda: binding.polyspec_verify_chain_greedy(data["models"], data["k"], draft, workspace=ws, out=out, device_status=status)
+    for _ in range(max(args.warmup, 3)):
+        call()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks = read_peaks()
+    elem = 4 if spec.dtype == torch.float32 else 2
+    vbytes = sum(int(m.shape[1]) for m in verifiers) * spec.B * spec.V * elem
+    tokens = verified_tokens(out["block_len"])
+    achieved = vbytes / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(args, spec) + ", greedy matching (verifier rows only)", "seed": args.seed},
+        "gpu_launches": 2 * args.steps, "mean_accepted_len_top_level": float(out["accepted_len"][0].float().mean()),
+        "roofline": {"bound": "hbm", "kernel": "stats_kernel in arg-max mode + greedy walk (whole call)", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                     "peak_source": f"of {peaks['source']}"},
+        "clocks": clocks}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -494,6 +549,8 @@ def main():
     ap.add_argument("--impl", default="polyspec", choices=["polyspec", "reference"])
     ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--sigma", type=float, default=1.0, help="inter-level noise of cfg5")
+    ap.add_argument("--rule", default="sampling", choices=["sampling", "greedy"],
+                    help="verification rule; greedy matching is timed on the logits-path workloads only")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
@@ -502,6 +559,8 @@ def main():
     spec = synth.FusedSpec() if args.workload == "cfg4" else chain_spec(args.workload, args.sigma)
     if args.impl == "reference":
         run_reference(args, spec)
+    elif args.rule == "greedy" and args.workload != "cfg4":
+        run_gpu_greedy(args, spec)
     elif args.workload == "cfg4":
         run_gpu_fused(args, spec)
     else:

@@ -181,6 +181,26 @@ polyspec_status polyspec_verify_from_hidden(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * polyspec_verify_chain_greedy -- the chain under greedy matching, the other verification rule
+ * Section 3.1 names and Section 4.5 compares with speculative sampling: a block token is accepted
+ * iff it is the verifier's most likely token at its position (first index on ties), the loop breaks
+ * at the first mismatch, and the token emitted after the accepted prefix is the verifier's most
+ * likely token there (at the first mismatch, or in the bonus row after a fully accepted block).
+ * No uniforms, no temperature; the emitted stream of a level is that verifier's own greedy text.
+ *
+ *   models, k, draft_tokens and the four outputs are those of polyspec_verify_chain; only the
+ *   verifiers models[0 .. n_models-2] are read (rows >= k[l] + 1); models[n_models-1].logits may be
+ *   NULL.  One pass over the verifiers' logits, no second pass.
+ */
+polyspec_status polyspec_verify_chain_greedy_workspace(int n_models, const int* k /* host */, const int* rows /* host [n_models] */,
+                                                       int B, int V, polyspec_dtype dt, size_t* bytes /* host out */);
+polyspec_status polyspec_verify_chain_greedy(
+    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */, const int32_t* draft_tokens,
+    int B, int V, polyspec_dtype dt,
+    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The two halves of polyspec_verify_from_hidden, for callers that want to time or overlap them:
  *   polyspec_from_hidden_project  both LM-head projections (one launch): logits and, from the same
  *                                 accumulators, every row's softmax-normaliser partials into the workspace;

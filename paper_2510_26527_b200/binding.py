@@ -26,6 +26,7 @@ EXPORTS = (
     "polyspec_verify_level_workspace", "polyspec_verify_level",
     "polyspec_verify_chain_workspace", "polyspec_verify_chain",
     "polyspec_chain_row_stats", "polyspec_chain_walk",
+    "polyspec_verify_chain_greedy_workspace", "polyspec_verify_chain_greedy",
     "polyspec_verify_chain_host_workspace", "polyspec_verify_chain_host",
     "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden", "polyspec_lm_head",
     "polyspec_from_hidden_project", "polyspec_from_hidden_verify",
@@ -72,6 +73,11 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_chain.restype = ci
     lib.polyspec_verify_chain.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, i32p, f32p, ci, ci, ci, cf,
                                           i32p, i32p, i32p, i32p, i32p, vp, sz, vp]
+    lib.polyspec_verify_chain_greedy_workspace.restype = ci
+    lib.polyspec_verify_chain_greedy_workspace.argtypes = [ci, cip, cip, ci, ci, ci, szp]
+    lib.polyspec_verify_chain_greedy.restype = ci
+    lib.polyspec_verify_chain_greedy.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, i32p, ci, ci, ci,
+                                                 i32p, i32p, i32p, i32p, i32p, vp, sz, vp]
     lib.polyspec_chain_row_stats.restype = ci
     lib.polyspec_chain_row_stats.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, i32p, vp, sz, vp]
     lib.polyspec_chain_walk.restype = ci
@@ -235,6 +241,48 @@ def polyspec_verify_chain(models, k, draft_tokens, uniforms, temperature, worksp
                                    _ptr(out["out_len"]), _ptr(device_status), _ptr(workspace), workspace.numel(),
                                    _stream(stream))
     _check(st, "polyspec_verify_chain")
+    out["device_status"] = device_status
+    return out
+
+
+def polyspec_verify_chain_greedy_workspace(k: Sequence[int], rows: Sequence[int], B: int, V: int, dt: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(load_library().polyspec_verify_chain_greedy_workspace(len(rows), _int_array(k), _int_array(rows), B, V, dt, ctypes.byref(n)),
+           "polyspec_verify_chain_greedy_workspace")
+    return n.value
+
+
+def polyspec_verify_chain_greedy(models, k, draft_tokens, workspace=None, out=None, device_status=None, stream=None):
+    """The chain under greedy matching.  models as in polyspec_verify_chain; the last entry (the drafter's logits)
+    is not read and may be None.  Returns the same four outputs plus the device status word."""
+    lib = load_library()
+    verifiers = list(models[:-1])
+    _dev_check(*verifiers, draft_tokens)
+    n = len(models)
+    L = n - 1
+    B, _, V = verifiers[0].shape
+    dt = _dt(verifiers[0])
+    rows = [int(m.shape[1]) for m in verifiers] + [int(k[-1])]
+    kmax = max(int(x) for x in k)
+    if any(m.dtype != verifiers[0].dtype or m.shape[0] != B or m.shape[2] != V for m in verifiers):
+        raise ValueError("all verifiers must share dtype, batch and vocabulary")
+    if tuple(draft_tokens.shape) != (B, int(k[-1])) or draft_tokens.dtype != torch.int32:
+        raise ValueError("draft_tokens must be int32 [B, k[-1]]")
+    dev = verifiers[0].device
+    if workspace is None:
+        workspace = _workspace(polyspec_verify_chain_greedy_workspace(k, rows, B, V, dt), dev)
+    if out is None:
+        out = chain_outputs(L, B, kmax, dev)
+    if device_status is None:
+        device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ptrs = [m.data_ptr() for m in verifiers] + [models[-1].data_ptr() if models[-1] is not None else None]
+    arr = (ModelLogits * n)(*[ModelLogits(pt, r) for pt, r in zip(ptrs, rows)])
+    with torch.cuda.device(dev):
+        st = lib.polyspec_verify_chain_greedy(arr, n, _int_array(k), _ptr(draft_tokens), B, V, dt,
+                                              _ptr(out["accepted_len"]), _ptr(out["block_len"]), _ptr(out["out_tokens"]),
+                                              _ptr(out["out_len"]), _ptr(device_status), _ptr(workspace), workspace.numel(),
+                                              _stream(stream))
+    _check(st, "polyspec_verify_chain_greedy")
     out["device_status"] = device_status
     return out
 

@@ -280,6 +280,94 @@ polyspec_status polyspec_chain_walk(
     return run_walk(a);
 }
 
+// ---- greedy matching: only the verifiers' rows are read (arg max), the drafter contributes its tokens
+namespace {
+polyspec_status greedy_shape(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt, long long* total_rows)
+{
+    if (n_models < 2 || n_models > kMaxModels || !k || !rows) return POLYSPEC_ERR_INVALID_ARG;
+    if (B <= 0 || V <= 0) return POLYSPEC_ERR_INVALID_ARG;
+    if (dt != POLYSPEC_F32 && dt != POLYSPEC_BF16) return POLYSPEC_ERR_INVALID_ARG;
+    if (V % 8 != 0 || V > kMaxV) return POLYSPEC_ERR_UNSUPPORTED;
+    long long acc = 0;
+    for (int l = 0; l < n_models - 1; ++l) {
+        if (k[l] < 1 || k[l] > kMaxK || rows[l] < k[l] + 1) return POLYSPEC_ERR_INVALID_ARG;
+        acc += static_cast<long long>(B) * rows[l];
+        if (acc > 0x3fffffffLL) return POLYSPEC_ERR_UNSUPPORTED;
+    }
+    if (plan_stats(acc, V, dt).n_items > 0x7fffffffLL) return POLYSPEC_ERR_UNSUPPORTED;
+    *total_rows = acc;
+    return POLYSPEC_OK;
+}
+}  // namespace
+
+polyspec_status polyspec_verify_chain_greedy_workspace(int n_models, const int* k, const int* rows, int B, int V,
+                                                       polyspec_dtype dt, size_t* bytes)
+{
+    if (!bytes) return POLYSPEC_ERR_INVALID_ARG;
+    long long total = 0;
+    polyspec_status st = greedy_shape(n_models, k, rows, B, V, dt, &total);
+    if (st != POLYSPEC_OK) return st;
+    *bytes = plan_stats(total, V, dt).partial_bytes;
+    return POLYSPEC_OK;
+}
+
+polyspec_status polyspec_verify_chain_greedy(
+    const polyspec_model_logits* models, int n_models, const int* k, const int32_t* draft_tokens,
+    int B, int V, polyspec_dtype dt,
+    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!models || !k || n_models < 2 || n_models > kMaxModels) return POLYSPEC_ERR_INVALID_ARG;
+    if (!draft_tokens || !accepted_len || !block_len || !out_tokens || !out_len) return POLYSPEC_ERR_INVALID_ARG;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return POLYSPEC_ERR_INVALID_ARG;
+    const int nv = n_models - 1;                    // verifiers; the drafter's logits are never read
+    int rows[kMaxModels];
+    const void* logits[kMaxModels];
+    for (int i = 0; i < n_models; ++i) { rows[i] = models[i].rows; logits[i] = models[i].logits; }
+    for (int l = 0; l < nv; ++l)
+        if (!logits[l] || !aligned16(logits[l])) return POLYSPEC_ERR_INVALID_ARG;
+    long long total = 0;
+    polyspec_status st = greedy_shape(n_models, k, rows, B, V, dt, &total);
+    if (st != POLYSPEC_OK) return st;
+    const StatsPlan pl = plan_stats(total, V, dt);
+    if (workspace_bytes < pl.partial_bytes) return POLYSPEC_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+    StatsParams sp;
+    if (fill_rows(sp.t, logits, rows, nv, B) < 0) return POLYSPEC_ERR_UNSUPPORTED;
+    sp.V = V;
+    sp.seg = pl.seg;
+    sp.parts = pl.parts;
+    sp.n_items = static_cast<int>(pl.n_items);
+    sp.c = 1.0f;
+    sp.partials = static_cast<float2*>(workspace);
+    sp.status = device_status;
+    if (launch_stats(dt, sp, s, /*argmax=*/true) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+
+    WalkParams wp;
+    std::memset(&wp, 0, sizeof wp);
+    wp.t = sp.t;
+    wp.V = V;
+    wp.parts = pl.parts;
+    wp.partials = sp.partials;
+    wp.n_levels = nv;
+    int kmax = 0;
+    for (int l = 0; l < kMaxLevels; ++l) {
+        wp.k[l] = l < nv ? k[l] : 0;
+        if (wp.k[l] > kmax) kmax = wp.k[l];
+    }
+    wp.kmax = kmax;
+    wp.B = B;
+    wp.draft_tokens = draft_tokens;
+    wp.accepted_len = accepted_len;
+    wp.block_len = block_len;
+    wp.out_tokens = out_tokens;
+    wp.out_len = out_len;
+    wp.device_status = device_status;
+    if (launch_greedy_walk(wp, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    return POLYSPEC_OK;
+}
+
 // Staging layout of the host-buffer call, after the partials: logits of each model, draft
 // tokens, uniforms, the four outputs, the status word; every piece 256-byte aligned.
 namespace {

@@ -81,8 +81,12 @@ struct StatsPlan {
 };
 StatsPlan plan_stats(long long total_rows, int V, polyspec_dtype dt);
 
-cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t stream);
+// argmax = true: the same pass produces arg-max partials (largest logit, index as int bits or -1)
+// for greedy matching instead of the softmax normaliser.
+cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t stream, bool argmax = false);
 cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p, cudaStream_t stream);
+// Greedy matching: reads arg-max partials (launch_stats with argmax = true) of the verifiers' rows only.
+cudaError_t launch_greedy_walk(const WalkParams& p, cudaStream_t stream);
 
 // LM-head projection on the tensor cores: out[r, v] = sum_d hidden[r, d] * W[v, d], bf16 inputs
 // (hidden [rows, d], W [V, d], both row-major and 16-byte aligned, d a multiple of 64), fp32

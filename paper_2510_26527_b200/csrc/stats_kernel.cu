@@ -132,7 +132,10 @@ __device__ __forceinline__ void cursor_open(const StatsParams& p, ChunkCursor& c
     cur.off = 0;
 }
 
-template <int DT>
+// MODE 0: softmax normaliser partials (E, s).  MODE 1: arg-max partials for greedy matching
+// (Section 3.1): (largest logit of the segment, index of its first occurrence as int bits; -1 if
+// the segment holds NaN or +inf).  Same pipeline, different arithmetic on the staged vectors.
+template <int DT, int MODE>
 __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsParams p)
 {
     using EL = Elems<DT>;
@@ -189,6 +192,12 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
         float s[kVecPerLane];
 #pragma unroll
         for (int u = 0; u < kVecPerLane; ++u) s[u] = 0.0f;
+        // arg-max state of this lane: its elements come in ascending index order, so a strictly
+        // larger value is always the first occurrence among the lane's own
+        float best = -INFINITY;
+        int best_at = 0x7fffffff;
+        uint32_t abs_max = 0;              // largest |bits|: above 0x7f800000 means a NaN went by
+        const int seg_first = (item % p.parts) * p.seg;      // row index of the segment's first element
 
         for (uint32_t off = 0; off < bytes; off += kChunkBytes, ++done) {
             __syncwarp();          // every lane has finished reading the stage the next copy will overwrite
@@ -212,24 +221,60 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
                 r[u] = (idx < nvec) ? ld_shared_v4(base + idx * 16) : EL::neg_inf();
             }
             float z[kVecPerLane][EPV];
-            float M = -INFINITY;
+            if (MODE == 0) {
+                float M = -INFINITY;
 #pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u) {
-                EL::unpack(r[u], z[u]);
+                for (int u = 0; u < kVecPerLane; ++u) {
+                    EL::unpack(r[u], z[u]);
 #pragma unroll
-                for (int e = 0; e < EPV; ++e) M = fmaxf(M, z[u][e]);
+                    for (int e = 0; e < EPV; ++e) M = fmaxf(M, z[u][e]);
+                }
+                const float En = (M == -INFINITY) ? kEmptyRef : ceilf(M * c);
+                if (En > E) {
+                    const float sc = pow2_neg(E - En);
+#pragma unroll
+                    for (int u = 0; u < kVecPerLane; ++u) s[u] *= sc;
+                    E = En;
+                }
+#pragma unroll
+                for (int u = 0; u < kVecPerLane; ++u)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) s[u] += ex2f(__fmaf_rn(z[u][e], c, -E));
+            } else {
+                constexpr int ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
+#pragma unroll
+                for (int u = 0; u < kVecPerLane; ++u) {
+                    EL::unpack(r[u], z[u]);
+                    float vm = z[u][0];
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        vm = fmaxf(vm, z[u][e]);
+                        abs_max = max(abs_max, __float_as_uint(z[u][e]) & 0x7fffffffu);
+                    }
+                    if (vm > best) {           // rare once the running maximum has settled
+                        best = vm;
+                        int e_first = 0;
+#pragma unroll
+                        for (int e = EPV - 1; e >= 0; --e) e_first = (z[u][e] == vm) ? e : e_first;
+                        best_at = seg_first + static_cast<int>(off / ELEM) + (lane + u * 32) * EPV + e_first;
+                    }
+                }
             }
-            const float En = (M == -INFINITY) ? kEmptyRef : ceilf(M * c);
-            if (En > E) {
-                const float sc = pow2_neg(E - En);
+        }
+
+        if (MODE == 1) {
+            // lanes -> warp: the larger value wins, equal values go to the lower index
 #pragma unroll
-                for (int u = 0; u < kVecPerLane; ++u) s[u] *= sc;
-                E = En;
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+                const int oa = __shfl_xor_sync(0xffffffffu, best_at, o);
+                const uint32_t om = __shfl_xor_sync(0xffffffffu, abs_max, o);
+                if (ov > best || (ov == best && oa < best_at)) { best = ov; best_at = oa; }
+                abs_max = max(abs_max, om);
             }
-#pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u)
-#pragma unroll
-                for (int e = 0; e < EPV; ++e) s[u] += ex2f(__fmaf_rn(z[u][e], c, -E));
+            const bool unusable = abs_max > 0x7f800000u || best == INFINITY;
+            if (lane == 0) p.partials[item] = make_float2(best, __int_as_float(unusable ? -1 : best_at));
+            continue;
         }
 
         // lanes -> warp: rebase every lane to the warp's largest reference (exact), then add
@@ -267,7 +312,7 @@ StatsPlan plan_stats(long long total_rows, int V, polyspec_dtype dt)
     return pl;
 }
 
-cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t stream)
+cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t stream, bool argmax)
 {
     if (p.n_items <= 0) return cudaSuccess;
     int dev = 0;
@@ -278,19 +323,24 @@ cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t s
         int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(stats_kernel<POLYSPEC_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kStatsSmemBytes));
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(stats_kernel<POLYSPEC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(kStatsSmemBytes));
-        if (e != cudaSuccess) return e;
+        const void* kernels[4] = {reinterpret_cast<const void*>(stats_kernel<POLYSPEC_F32, 0>),
+                                  reinterpret_cast<const void*>(stats_kernel<POLYSPEC_BF16, 0>),
+                                  reinterpret_cast<const void*>(stats_kernel<POLYSPEC_F32, 1>),
+                                  reinterpret_cast<const void*>(stats_kernel<POLYSPEC_BF16, 1>)};
+        for (const void* k : kernels) {
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kStatsSmemBytes));
+            if (e != cudaSuccess) return e;
+        }
         g_sm_count[dev] = sms > 0 ? sms : 148;
     }
     const int grid = p.n_items < g_sm_count[dev] ? p.n_items : g_sm_count[dev];   // one CTA per SM
-    if (dt == POLYSPEC_BF16)
-        stats_kernel<POLYSPEC_BF16><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
-    else
-        stats_kernel<POLYSPEC_F32><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
+    if (dt == POLYSPEC_BF16) {
+        if (argmax) stats_kernel<POLYSPEC_BF16, 1><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
+        else stats_kernel<POLYSPEC_BF16, 0><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
+    } else {
+        if (argmax) stats_kernel<POLYSPEC_F32, 1><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
+        else stats_kernel<POLYSPEC_F32, 0><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
+    }
     return cudaGetLastError();
 }
 
