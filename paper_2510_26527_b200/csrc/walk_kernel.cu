@@ -386,6 +386,7 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
     __shared__ RowStat st_p[kMaxK + 1];
     __shared__ RowStat st_q[kMaxK + 1];
     __shared__ int sh_a, sh_bad;
+    __shared__ float g_zp[32], g_zq[32], g_u[32];       // logits at the block tokens, accept uniforms
     __shared__ SampleShared sh_sample;
 
     constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
@@ -424,7 +425,23 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
         const char* base_p = static_cast<const char*>(p.t.logits[l]) + static_cast<size_t>(b) * p.t.rows[l] * row_bytes;
         const char* base_q = static_cast<const char*>(p.t.logits[l + 1]) + static_cast<size_t>(b) * p.t.rows[l + 1] * row_bytes;
 
-        // 1. normalisers of p rows 0..m and q rows 0..m-1
+        // 1. normalisers of p rows 0..m and q rows 0..m-1; the last warp first requests the logits at the
+        // block tokens and the accept uniforms, so that those loads are in flight during the merges
+        if ((tid >> 5) == kWalkWarps - 1) {
+            const int j = tid & 31;
+            float zp = 0.0f, zq = 0.0f, uu = 0.0f;
+            if (j < m) {
+                const int x = tok[j];
+                if (x >= 0 && x < p.V) {
+                    zp = load_logit<DT>(base_p + j * row_bytes, x);
+                    zq = load_logit<DT>(base_q + j * row_bytes, x);
+                }
+                uu = p.uniforms[lb * (p.kmax + 1) + j];
+            }
+            g_zp[j] = zp;
+            g_zq[j] = zq;
+            g_u[j] = uu;
+        }
         for (int r = tid >> 5; r < 2 * m + 1; r += kWalkWarps) {          // one warp per row
             const bool is_q = r > m;
             const int j = is_q ? r - (m + 1) : r;
@@ -443,11 +460,10 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
                 if (x < 0 || x >= p.V || !stat_ok(sp) || !stat_ok(sq)) {
                     bad = true;
                 } else {
-                    const float zp = load_logit<DT>(base_p + tid * row_bytes, x);
-                    const float zq = load_logit<DT>(base_q + tid * row_bytes, x);
+                    const float zp = g_zp[tid], zq = g_zq[tid];
                     const double P = exp2(static_cast<double>(zp) * cd - static_cast<double>(sp.E)) / sp.Z;
                     const double Q = exp2(static_cast<double>(zq) * cd - static_cast<double>(sq.E)) / sq.Z;
-                    const double u = static_cast<double>(p.uniforms[lb * (p.kmax + 1) + tid]);
+                    const double u = static_cast<double>(g_u[tid]);
                     rej = !(u * Q <= P);
                     pf = static_cast<float>(P);
                     qf = static_cast<float>(Q);
