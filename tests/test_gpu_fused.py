@@ -125,3 +125,19 @@ def test_fused_config4_full(oracle):
     d = synth.make_fused(spec, seed=0, device=DEV)
     got, ora = _fused_compare(oracle, d, lambda dl: 4 * dl / spec.temperature)
     assert 0.5 < ora["accepted_len"].mean() < spec.k
+
+
+def test_halves_of_the_fused_call_equal_the_whole_call():
+    spec = synth.FusedSpec(B=8, k=4, V=2048, d_p=256, d_q=128)
+    d = synth.make_fused(spec, seed=5, device=DEV)
+    whole = binding.polyspec_verify_from_hidden(d["hidden_p"], d["W_p"], d["hidden_q"], d["W_q"], d["draft_tokens"],
+                                                d["uniforms"], d["temperature"])
+    call = binding.FusedCall(d["hidden_p"], d["W_p"], d["hidden_q"], d["W_q"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    call.project()
+    halves = call.verify()
+    torch.cuda.synchronize()
+    assert torch.equal(halves["accepted_len"], whole["accepted_len"]) and torch.equal(halves["next_token"], whole["next_token"])
+    again = call.launch()
+    torch.cuda.synchronize()
+    assert torch.equal(again["accepted_len"], whole["accepted_len"]) and torch.equal(again["next_token"], whole["next_token"])
+    assert int(call.device_status.item()) == 0

@@ -312,3 +312,17 @@ def test_chain_batch_sizes_across_the_cluster_thresholds(oracle, B):
     ora = _oracle_chain(oracle, d)
     counts, bad = H.compare_chain(out, ora)
     _assert_parity(counts, bad, B * sum(spec.k), f"cfg3 recipe at B={B}")
+
+
+def test_halves_of_the_chain_call_equal_the_whole_call():
+    spec = synth.scaled(synth.config("cfg5", sigma=0.5), B=10, V=12288)
+    d = synth.make_chain(spec, seed=21, device=DEV)
+    whole = _run_chain(d)
+    call = binding.ChainCall(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    call.row_stats()
+    halves = _np(call.walk())
+    for key in ("accepted_len", "block_len", "out_tokens", "out_len"):
+        assert (halves[key] == whole[key]).all()
+    again = _np(call.launch())
+    for key in ("accepted_len", "block_len", "out_tokens", "out_len"):
+        assert (again[key] == whole[key]).all()
