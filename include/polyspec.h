@@ -231,6 +231,25 @@ polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, in
                                  int32_t* device_status, void* cuda_stream);
 
 /*
+ * Cost model of Section 3.2 (host arithmetic only; nothing is launched).
+ *
+ * polyspec_cost_total_time -- Lemma 3.1 (Eq. 3): the time to generate N tokens with n models,
+ *     T = sum_{i=1}^{n-1} (N / L_i) T_i + beta (N / L_{n-1}) T_n,
+ *   T[0..n-1] the forward-pass costs T_1..T_n, L[0..n-2] the acceptance lengths L_1..L_{n-1} (Eq. 1:
+ *   what polyspec_verify_chain reports as accepted_len, averaged), beta the drafter's scaling factor.
+ *   Returns NaN for n < 2, a NULL array or a non-positive L.
+ * polyspec_cost_insertion -- Theorem 3.2, first condition, with the quantities of Table 1: inserting
+ *   M_new between M_i and M_{i+1} pays off iff
+ *     T_new / T_i  <  L_new (1 / L_i - 1 / L_{i-new}),
+ *   L_i the acceptance length of the pair (M_i, M_{i+1}) before the insertion, L_{i-new} that of
+ *   (M_i, M_new) and L_new that of (M_new, M_{i+1}) after it.  Writes both sides (either pointer may be
+ *   NULL) and returns 1 if the condition holds, 0 if not, -1 on non-positive inputs.
+ */
+double polyspec_cost_total_time(int n, const double* T /* host [n] */, const double* L /* host [n-1] */, double beta, double N);
+int polyspec_cost_insertion(double T_new, double T_i, double L_new, double L_i, double L_i_new,
+                            double* lhs /* host out */, double* rhs /* host out */);
+
+/*
  * polyspec_verify_level_static -- polyspec_verify_level without a workspace argument.
  * (The paper has no counterpart to this call; it exists for integration reasons only.)
  *

@@ -31,6 +31,7 @@ EXPORTS = (
     "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden", "polyspec_lm_head",
     "polyspec_from_hidden_project", "polyspec_from_hidden_verify",
     "polyspec_static_scratch_bytes", "polyspec_verify_level_static",
+    "polyspec_cost_total_time", "polyspec_cost_insertion",
 )
 
 
@@ -98,6 +99,10 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_from_hidden_verify.argtypes = [ci, i32p, f32p, i32p, ci, ci, ci, ci, ci, cf, i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
     lib.polyspec_lm_head.restype = ci
     lib.polyspec_lm_head.argtypes = [vp, vp, ci, ci, ci, f32p, i32p, vp]
+    lib.polyspec_cost_total_time.restype = ctypes.c_double
+    lib.polyspec_cost_total_time.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), ctypes.c_double, ctypes.c_double]
+    lib.polyspec_cost_insertion.restype = ci
+    lib.polyspec_cost_insertion.argtypes = [ctypes.c_double] * 5 + [ctypes.POINTER(ctypes.c_double)] * 2
     lib.polyspec_static_scratch_bytes.restype = sz
     lib.polyspec_static_scratch_bytes.argtypes = []
     lib.polyspec_verify_level_static.restype = ci
@@ -513,3 +518,24 @@ def polyspec_verify_level_static(logits_p, logits_q, draft_tokens, uniforms, tem
             _ptr(out.get("p_at_draft")), _ptr(out.get("q_at_draft")), _ptr(device_status), _stream(stream))
     _check(st, "polyspec_verify_level_static")
     return out
+
+
+# ------------------------------------------------------------------ cost model (host arithmetic)
+def polyspec_cost_total_time(T: Sequence[float], L: Sequence[float], beta: float, N: float) -> float:
+    """Lemma 3.1 (Eq. 3): T = sum_{i<n} (N / L_i) T_i + beta (N / L_{n-1}) T_n."""
+    n = len(T)
+    if len(L) != n - 1:
+        raise ValueError("L must hold n - 1 acceptance lengths")
+    Ta = (ctypes.c_double * n)(*[float(x) for x in T])
+    La = (ctypes.c_double * max(n - 1, 1))(*[float(x) for x in L])
+    return float(load_library().polyspec_cost_total_time(n, Ta, La, float(beta), float(N)))
+
+
+def polyspec_cost_insertion(T_new: float, T_i: float, L_new: float, L_i: float, L_i_new: float):
+    """Theorem 3.2, first condition: (improves, T_new / T_i, L_new (1 / L_i - 1 / L_{i-new}))."""
+    lhs, rhs = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    r = load_library().polyspec_cost_insertion(float(T_new), float(T_i), float(L_new), float(L_i), float(L_i_new),
+                                               ctypes.byref(lhs), ctypes.byref(rhs))
+    if r < 0:
+        raise ValueError("all five quantities must be positive")
+    return bool(r), lhs.value, rhs.value

@@ -280,6 +280,28 @@ polyspec_status polyspec_chain_walk(
     return run_walk(a);
 }
 
+// ---- cost model of Section 3.2 (host arithmetic)
+double polyspec_cost_total_time(int n, const double* T, const double* L, double beta, double N)
+{
+    if (n < 2 || !T || !L) return std::nan("");
+    double total = 0.0;
+    for (int i = 0; i < n - 1; ++i) {
+        if (!(L[i] > 0.0)) return std::nan("");
+        total += N / L[i] * T[i];
+    }
+    return total + beta * (N / L[n - 2]) * T[n - 1];
+}
+
+int polyspec_cost_insertion(double T_new, double T_i, double L_new, double L_i, double L_i_new, double* lhs, double* rhs)
+{
+    if (!(T_i > 0.0) || !(T_new > 0.0) || !(L_new > 0.0) || !(L_i > 0.0) || !(L_i_new > 0.0)) return -1;
+    const double a = T_new / T_i;
+    const double b = L_new * (1.0 / L_i - 1.0 / L_i_new);
+    if (lhs) *lhs = a;
+    if (rhs) *rhs = b;
+    return a < b ? 1 : 0;
+}
+
 // ---- greedy matching: only the verifiers' rows are read (arg max), the drafter contributes its tokens
 namespace {
 polyspec_status greedy_shape(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt, long long* total_rows)
