@@ -21,7 +21,6 @@
 // Warp roles in each CTA:
 //   warp 0      TMA producer (one elected lane issues).  Both CTAs load their own tiles; all copies of a stage
 //               complete on the leader CTA's "full" barrier (no multicast anywhere)
-//   warp 10     L2 prefetch of W: 1 KiB contiguous per row, a few K blocks ahead of the TMA loads
 //   warp 1      MMA issuer (one elected lane, leader CTA only); allocates / frees TMEM in both CTAs.
 //               tcgen05.commit arrives on the "empty" / "accumulator full" barriers of both CTAs
 //   warps 2..9  epilogue (two warps per TMEM lane quarter, alternate 16-column chunks): TMEM ->
@@ -55,10 +54,7 @@ constexpr int kBytesA = kTileV * kBlockK * 2;                // 16 KiB: this CTA
 constexpr int kBytesBMax = (kMaxCols / 2) * kBlockK * 2;     // 18 KiB: this CTA's half of the hidden tile
 constexpr int kStageBytes = kBytesA + kBytesBMax;            // 34 KiB
 constexpr int kEpiWarps = 8;                // warps 2..9: two per TMEM lane quarter, alternating 16-column chunks
-constexpr int kPrefetchWarp = 2 + kEpiWarps;
-constexpr int kGemmThreads = 32 * (kPrefetchWarp + 1);
-constexpr int kPrefetchK = 8;               // K blocks per L2 prefetch: 1 KiB contiguous per W row
-constexpr int kPrefetchLead = 16;           // how many K blocks the prefetch may run ahead of the TMA loads
+constexpr int kGemmThreads = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinLimitG = 1u << 20;
 constexpr int kScratchPitch = 32;                            // an epilogue warp's staging tile: [16 hidden rows][32 vocabulary entries] fp32
@@ -69,7 +65,6 @@ struct GemmJob {
     CUtensorMap map_w;      // [V, d] bf16, box {64, 128}
     CUtensorMap map_h;      // [rows, d] bf16, box {64, chunk / 2}
     CUtensorMap map_out;    // [rows, V] fp32, box {32, 16}, no swizzle: the epilogue's stores
-    const char* w;          // W itself, for the L2 prefetch that runs ahead of the TMA loads
     float* out;             // [rows, V]
     float2* partials;       // [rows, parts] row statistics of the tile just computed, or nullptr
     int rows;
@@ -277,7 +272,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ uint32_t loads_issued;       // K blocks the TMA producer has issued so far
 
     // broadcast from lane 0 so that the compiler knows the role branches and everything derived
     // from them (ring positions, descriptors) are warp-uniform
@@ -302,7 +296,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        loads_issued = 0;
         for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
         for (int a = 0; a < 2; ++a) mbar_init(acc_full + 8u * a, 1);
         for (int a = 0; a < 3; ++a) mbar_init(slot_empty + 8u * a, 2 * kEpiWarps);
@@ -344,7 +337,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
                     tma_load_2d(a_dst, &job.map_w, kb * kBlockK, w_row, bar);
                     tma_load_2d(a_dst + kBytesA, &job.map_h, kb * kBlockK, h_row, bar);
                     if (two) tma_load_2d(a_dst + kBytesA + half * (kBlockK * 2), &job.map_h, kb * kBlockK, h_row + job.chunk, bar);
-                    *reinterpret_cast<volatile uint32_t*>(&loads_issued) = it + 1;
                 }
                 __syncwarp();
                 if (++stage == kStagesG) { stage = 0; phase ^= 1u; }
@@ -360,39 +352,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             const uint32_t b = (rank == 0 ? full_bar : empty_bar) + 8u * (q % kStagesG);
             for (uint32_t i = 0; i < kSpinLimitG; ++i)
                 if (mbar_try(b, (q / kStagesG) & 1u) || *abort_p) break;
-        }
-    } else if (warp == kPrefetchWarp) {
-        // ------------------------------------------------------------------ L2 prefetch of W (both CTAs)
-        // A TMA box touches 128 bytes in each of 128 rows of W that lie d * 2 bytes apart: 128 DRAM
-        // pages per K block, each page visited again only a K block later.  This warp runs a little
-        // ahead and asks L2 for 1 KiB contiguous per row (8 K blocks at once), so DRAM sees page-long
-        // bursts and the TMA loads find their lines in L2.
-        uint32_t it = 0;
-        bool live = true;
-        for (int item = first_item; live && item >= 0 && item < p.total_items; item += item_step) {
-            int j, vt, nb;
-            decode_item(p, item, &j, &vt, &nb);
-            const GemmJob& job = p.job[j];
-            const size_t row_bytes = static_cast<size_t>(job.kblocks) * (kBlockK * 2);
-            const int v0 = vt * kPairV + static_cast<int>(rank) * kTileV;
-            for (int kb = 0; live && kb < job.kblocks; kb += kPrefetchK) {
-                uint32_t spins = 0;
-                while (*reinterpret_cast<volatile uint32_t*>(&loads_issued) + kPrefetchLead < it) {
-                    __nanosleep(64);
-                    if (*abort_p || ++spins > (1u << 22)) { live = false; break; }
-                }
-                if (!live) break;
-                const int nk = min(kPrefetchK, job.kblocks - kb);
-                it += nk;
-#pragma unroll
-                for (int q = 0; q < kTileV / 32; ++q) {
-                    const int v = v0 + q * 32 + lane;
-                    if (v < p.V) {
-                        const char* src = job.w + static_cast<size_t>(v) * row_bytes + static_cast<size_t>(kb) * (kBlockK * 2);
-                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(nk * kBlockK * 2) : "memory");
-                    }
-                }
-            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
@@ -665,7 +624,6 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
         job.kblocks = pr.d / kBlockK;
         job.out = pr.out;
         job.partials = pr.partials;
-        job.w = static_cast<const char*>(pr.W);
         job.items = p.vtiles * job.nblocks;
         p.total_items += job.items;
         if (!encode_map(&job.map_w, pr.W, V, pr.d, kTileV)) return cudaErrorInvalidValue;
