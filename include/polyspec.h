@@ -73,6 +73,9 @@ typedef enum { POLYSPEC_F32 = 0, POLYSPEC_BF16 = 1 } polyspec_dtype;
 const char* polyspec_status_string(polyspec_status s);
 /* major * 10000 + minor * 100 + patch */
 int polyspec_version(void);
+/* The CUDA runtime's message for the most recent call that returned POLYSPEC_ERR_CUDA ("no error" if none did).
+ * Static string; not synchronised between host threads. */
+const char* polyspec_last_cuda_error(void);
 
 /*
  * polyspec_verify_level -- one adjacent pair (verifier p, drafter-side q) over a batch of

@@ -22,7 +22,7 @@ F32, BF16 = 0, 1
 MAX_K, MAX_MODELS = 32, 8
 
 EXPORTS = (
-    "polyspec_status_string", "polyspec_version",
+    "polyspec_status_string", "polyspec_version", "polyspec_last_cuda_error",
     "polyspec_verify_level_workspace", "polyspec_verify_level",
     "polyspec_verify_chain_workspace", "polyspec_verify_chain",
     "polyspec_chain_row_stats", "polyspec_chain_walk",
@@ -38,7 +38,10 @@ EXPORTS = (
 class PolyspecError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {status_string(status)} (status {status})")
+        detail = ""
+        if status == ERR_CUDA and _lib is not None:
+            detail = ": " + _lib.polyspec_last_cuda_error().decode()
+        super().__init__(f"{where}: {status_string(status)} (status {status}){detail}")
 
 
 class ModelLogits(ctypes.Structure):
@@ -62,6 +65,8 @@ def load_library() -> ctypes.CDLL:
     szp, cip = ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_int)
     lib.polyspec_status_string.restype = ctypes.c_char_p
     lib.polyspec_status_string.argtypes = [ci]
+    lib.polyspec_last_cuda_error.restype = ctypes.c_char_p
+    lib.polyspec_last_cuda_error.argtypes = []
     lib.polyspec_version.restype = ci
     lib.polyspec_version.argtypes = []
     lib.polyspec_verify_level_workspace.restype = ci

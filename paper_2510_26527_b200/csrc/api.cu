@@ -11,6 +11,15 @@ namespace {
 
 constexpr double kLog2e = 1.4426950408889634074;
 
+// The runtime's code for the most recent POLYSPEC_ERR_CUDA (see polyspec_last_cuda_error).
+cudaError_t g_last_cuda_error = cudaSuccess;
+inline bool cuda_failed(cudaError_t e)
+{
+    if (e == cudaSuccess) return false;
+    g_last_cuda_error = e;
+    return true;
+}
+
 inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t elem_size(polyspec_dtype dt) { return dt == POLYSPEC_BF16 ? 2 : 4; }
@@ -110,7 +119,7 @@ polyspec_status run_stats(const ChainArgs& a)
     StatsParams sp;
     polyspec_status st = prepare_chain(a, &pl, &sp);
     if (st != POLYSPEC_OK) return st;
-    if (launch_stats(a.dt, sp, a.stream) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(launch_stats(a.dt, sp, a.stream))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
@@ -147,7 +156,7 @@ polyspec_status run_walk(const ChainArgs& a)
     wp.p_at = a.p_at;
     wp.q_at = a.q_at;
     wp.device_status = a.device_status;
-    if (launch_walk(a.dt, wp, a.stream) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(launch_walk(a.dt, wp, a.stream))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
@@ -193,6 +202,8 @@ const char* polyspec_status_string(polyspec_status s)
 }
 
 int polyspec_version(void) { return 100; }
+
+const char* polyspec_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 polyspec_status polyspec_verify_level_workspace(int B, int k, int V, polyspec_dtype dt, size_t* bytes)
 {
@@ -364,7 +375,7 @@ polyspec_status polyspec_verify_chain_greedy(
     sp.c = 1.0f;
     sp.partials = static_cast<float2*>(workspace);
     sp.status = device_status;
-    if (launch_stats(dt, sp, s, /*argmax=*/true) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(launch_stats(dt, sp, s, /*argmax=*/true))) return POLYSPEC_ERR_CUDA;
 
     WalkParams wp;
     std::memset(&wp, 0, sizeof wp);
@@ -386,7 +397,7 @@ polyspec_status polyspec_verify_chain_greedy(
     wp.out_tokens = out_tokens;
     wp.out_len = out_len;
     wp.device_status = device_status;
-    if (launch_greedy_walk(wp, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(launch_greedy_walk(wp, s))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
@@ -466,9 +477,9 @@ polyspec_status polyspec_verify_chain_host(
         dev_models[i].logits = ws + h.logits[i];
         dev_models[i].rows = rows[i];
     }
-    if (cudaMemcpyAsync(ws + h.tokens, draft_tokens_host, h.tokens_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (cudaMemcpyAsync(ws + h.uniforms, uniforms_host, h.uniforms_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (cudaMemsetAsync(ws + h.status, 0, 4, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemcpyAsync(ws + h.tokens, draft_tokens_host, h.tokens_bytes, cudaMemcpyHostToDevice, s))) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemcpyAsync(ws + h.uniforms, uniforms_host, h.uniforms_bytes, cudaMemcpyHostToDevice, s))) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemsetAsync(ws + h.status, 0, 4, s))) return POLYSPEC_ERR_CUDA;
 
     st = polyspec_verify_chain(dev_models, n_models, k,
                                reinterpret_cast<const int32_t*>(ws + h.tokens), reinterpret_cast<const float*>(ws + h.uniforms),
@@ -477,11 +488,11 @@ polyspec_status polyspec_verify_chain_host(
                                reinterpret_cast<int32_t*>(ws + h.otok), reinterpret_cast<int32_t*>(ws + h.olen),
                                reinterpret_cast<int32_t*>(ws + h.status), ws + h.partials, h.logits[0] - h.partials, s);
     if (st != POLYSPEC_OK) return st;
-    if (cudaMemcpyAsync(accepted_len_host, ws + h.acc, h.lb_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (cudaMemcpyAsync(block_len_host, ws + h.blk, h.lb_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (cudaMemcpyAsync(out_len_host, ws + h.olen, h.lb_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (cudaMemcpyAsync(out_tokens_host, ws + h.otok, h.otok_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
-    if (host_status && cudaMemcpyAsync(host_status, ws + h.status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemcpyAsync(accepted_len_host, ws + h.acc, h.lb_bytes, cudaMemcpyDeviceToHost, s))) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemcpyAsync(block_len_host, ws + h.blk, h.lb_bytes, cudaMemcpyDeviceToHost, s))) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemcpyAsync(out_len_host, ws + h.olen, h.lb_bytes, cudaMemcpyDeviceToHost, s))) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(cudaMemcpyAsync(out_tokens_host, ws + h.otok, h.otok_bytes, cudaMemcpyDeviceToHost, s))) return POLYSPEC_ERR_CUDA;
+    if (host_status && cuda_failed(cudaMemcpyAsync(host_status, ws + h.status, 4, cudaMemcpyDeviceToHost, s))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
@@ -492,7 +503,7 @@ polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, in
     if (!aligned16(hidden) || !aligned16(W) || !aligned16(logits)) return POLYSPEC_ERR_INVALID_ARG;
     if (d % 64 != 0 || V % 4 != 0 || static_cast<long long>(rows) * V > 0x7fffffffLL * 16) return POLYSPEC_ERR_UNSUPPORTED;
     const LmHeadProblem pr = {hidden, W, rows, d, logits, nullptr};
-    if (launch_lmhead(&pr, 1, V, 0.0f, device_status, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(launch_lmhead(&pr, 1, V, 0.0f, device_status, static_cast<cudaStream_t>(cuda_stream)))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
@@ -571,7 +582,7 @@ polyspec_status polyspec_from_hidden_project(
     const LmHeadProblem probs[2] = {{hidden_p, W_p, B * (k + 1), d_p, c.lp, partials},
                                     {hidden_q, W_q, B * rows_q, d_q, c.lq, partials + static_cast<size_t>(B) * (k + 1) * parts}};
     const float scale = static_cast<float>(kLog2e / static_cast<double>(temperature));
-    if (launch_lmhead(probs, 2, V, scale, device_status, c.s) != cudaSuccess) return POLYSPEC_ERR_CUDA;
+    if (cuda_failed(launch_lmhead(probs, 2, V, scale, device_status, c.s))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 

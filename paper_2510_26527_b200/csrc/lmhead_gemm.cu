@@ -11,7 +11,8 @@
 //     so each SM fills and reads only half of it;
 //   - d is the K loop in blocks of 64 elements = one 128-byte swizzle row; both operands are
 //     K-major in shared memory exactly as 2-D TMA with 128-byte swizzle writes them; a
-//     6-stage ring of (W tile, hidden half-tile) keeps about 200 KiB in flight per SM;
+//     5-stage ring of (W tile, hidden half-tile) keeps about 170 KiB in flight per SM (a sixth
+//     stage measured no faster);
 //   - the accumulator lives in TMEM (lane = vocabulary entry, column = hidden row) and is
 //     read back with tcgen05.ld by four epilogue warps per CTA.
 //
@@ -27,7 +28,7 @@
 //               registers -> a 2 KiB staging tile per warp -> global by 2-D TMA store; all sixteen
 //               epilogue warps of the pair arrive on the leader's "accumulator empty" barrier.
 //               On request the epilogue also emits the row statistics of the tile (the softmax
-//               normaliser partial of each hidden row over each warp's 32 vocabulary entries, in the
+//               normaliser partial of each hidden row over the CTA's 128 vocabulary entries, in the
 //               format of the row-statistics kernel), so the logits need no second pass for them
 // TMEM holds more than one accumulator so that the epilogue of a tile overlaps the K loop of the
 // next: two slots of 256 columns when every column block fits one, else three slots of 144 columns
@@ -49,7 +50,7 @@ constexpr int kPairV = 2 * kTileV;          // vocabulary entries per CTA pair a
 constexpr int kBlockK = 64;                 // bf16 elements per K block (one 128-byte swizzle row)
 constexpr int kMmaK = 16;                   // K of one tcgen05.mma for 16-bit inputs
 constexpr int kMaxCols = 288;               // widest column block (TMEM columns per accumulator)
-constexpr int kStagesG = 6;
+constexpr int kStagesG = 5;                   // a sixth stage measured no faster (and the space now holds the statistics)
 constexpr int kBytesA = kTileV * kBlockK * 2;                // 16 KiB: this CTA's rows of W
 constexpr int kBytesBMax = (kMaxCols / 2) * kBlockK * 2;     // 18 KiB: this CTA's half of the hidden tile
 constexpr int kStageBytes = kBytesA + kBytesBMax;            // 34 KiB
@@ -59,7 +60,8 @@ constexpr int kTmemCols = 512;
 constexpr uint32_t kSpinLimitG = 1u << 20;
 constexpr int kScratchPitch = 32;                            // an epilogue warp's staging tile: [16 hidden rows][32 vocabulary entries] fp32
 constexpr int kStatStageBytes = kEpiWarps * 16 * kScratchPitch * 4;
-constexpr size_t kGemmSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStagesG) * kStageBytes + 256 /* barriers */ + kStatStageBytes;
+constexpr int kStatMergeBytes = 4 * kMaxCols * 8;            // (E, s) of every column from each of the four lane quarters
+constexpr size_t kGemmSmemBytes = 1024 /* alignment slack */ + static_cast<size_t>(kStagesG) * kStageBytes + 256 /* barriers */ + kStatStageBytes + kStatMergeBytes;
 
 struct GemmJob {
     CUtensorMap map_w;      // [V, d] bf16, box {64, 128}
@@ -86,7 +88,7 @@ struct GemmParams {
     // consecutive ones (round robin), one per MMA chunk: 2 slots of 256, 1 per tile when every column
     // block fits 256 columns, else 3 slots of 144, 2 per tile
     int n_slots, slots_per_tile, slot_cols;
-    int parts;              // 32-entry vocabulary slices per row = 8 * vtiles (row statistics)
+    int parts;              // 128-entry vocabulary slices per row = 2 * vtiles (row statistics)
     float c;                // log2(e) / T (row statistics)
     int32_t* status;
 };
@@ -244,6 +246,10 @@ __device__ __forceinline__ float pow2_neg(float d)
 {
     return (d < -126.0f) ? 0.0f : __int_as_float((static_cast<int>(d) + 127) << 23);
 }
+__device__ __forceinline__ void mbar_arrive_local(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Work item -> (job, vocabulary tile, column block).  Items of job 0 come first; inside a job
@@ -293,12 +299,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
     const uint32_t full_bar = bars, empty_bar = full_bar + 8u * kStagesG;       // full: used in the leader only
     const uint32_t acc_full = empty_bar + 8u * kStagesG, slot_empty = acc_full + 16u;   // slot_empty[3]: leader only
     float* stat_scratch = reinterpret_cast<float*>(smem_dyn + (bars - raw) + 256);     // per epilogue warp [16][kScratchPitch]
+    float2* stat_merge = reinterpret_cast<float2*>(smem_dyn + (bars - raw) + 256 + kStatStageBytes);   // [4][kMaxCols]
+    const uint32_t epi_bar = slot_empty + 24u;      // the epilogue warps of this CTA meet here (bounded, unlike bar.sync)
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s = 0; s < kStagesG; ++s) { mbar_init(full_bar + 8u * s, 1); mbar_init(empty_bar + 8u * s, 1); }
         for (int a = 0; a < 2; ++a) mbar_init(acc_full + 8u * a, 1);
         for (int a = 0; a < 3; ++a) mbar_init(slot_empty + 8u * a, 2 * kEpiWarps);
+        mbar_init(epi_bar, kEpiWarps);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -403,7 +412,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
         const int half_id = (warp - 2) >> 2;            // which of the quarter's two warps this is
         const uint32_t leader_slot_empty = cluster_addr(slot_empty, 0);
         float* scratch = stat_scratch + (warp - 2) * (16 * kScratchPitch);
-        uint32_t tile_n = 0;
+        uint32_t tile_n = 0, epi_phase = 0;
         bool ok = true;
         for (int item = first_item; ok && item >= 0 && item < p.total_items; item += item_step, ++tile_n) {
             int j, vt, nb;
@@ -422,7 +431,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
             };
             bool freed0 = p.slots_per_tile == 1;        // slot0 handed back already (or is the only, last one)
             const bool stats = job.partials != nullptr;
-            const int slice = (vt * 2 + static_cast<int>(rank)) * 4 + quarter;      // this warp's 32-entry slice of the row
+            const int slice = vt * 2 + static_cast<int>(rank);      // this CTA's 128-entry slice of the row
             // the two warps of a quarter take alternate 16-column chunks; a warp's next chunk is already
             // on its way from TMEM while it works on the current one
             uint32_t nxt[16];
@@ -474,14 +483,37 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
                     const float lo = (lane & 16) ? s2 : sm, hi = (lane & 16) ? sm : s2;       // same order in both lanes
                     const float Elo = (lane & 16) ? E2 : E, Ehi = (lane & 16) ? E : E2;
                     const float tot = __fadd_rn(__fmul_rn(lo, pow2_neg(Elo - Em)), __fmul_rn(hi, pow2_neg(Ehi - Em)));
-                    const int row = row0 + c0 + col;
-                    if (lane < 16 && row < job.rows) job.partials[static_cast<size_t>(row) * p.parts + slice] = make_float2(Em, tot);
+                    if (lane < 16) stat_merge[quarter * kMaxCols + c0 + col] = make_float2(Em, tot);
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (!freed0 && lane == 0) mbar_arrive_cluster(leader_slot_empty + 8u * slot0);     // (a warp without chunks in slot1)
             if (lane == 0) mbar_arrive_cluster(leader_slot_empty + 8u * slot1);     // the accumulator may be overwritten
+            if (stats) {
+                // all chunks are in: merge the four quarters of every column into the partial of this CTA's slice
+                __syncwarp();
+                if (lane == 0) mbar_arrive_local(epi_bar);
+                if (!mbar_wait(epi_bar, epi_phase, abort_p)) { ok = false; break; }
+                epi_phase ^= 1u;
+                for (int col = (warp - 2) * 32 + lane; col < job.block_cols; col += 32 * kEpiWarps) {
+                    const int row = row0 + col;
+                    if (row < job.rows) {
+                        float2 q[4];
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) q[w] = stat_merge[w * kMaxCols + col];
+                        const float Em = fmaxf(fmaxf(q[0].x, q[1].x), fmaxf(q[2].x, q[3].x));
+                        float tot = 0.0f;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) tot = __fadd_rn(tot, __fmul_rn(q[w].y, pow2_neg(q[w].x - Em)));
+                        job.partials[static_cast<size_t>(row) * p.parts + slice] = make_float2(Em, tot);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive_local(epi_bar);
+                if (!mbar_wait(epi_bar, epi_phase, abort_p)) { ok = false; break; }     // the merge area may be rewritten
+                epi_phase ^= 1u;
+            }
         }
         if (lane == 0) tma_store_wait_all();        // this thread's stores have landed before the CTA may exit
         if (!ok && lane == 0) raise_abort(&abort_flag, peer, p.status);
@@ -587,7 +619,7 @@ cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int
     p.n_jobs = n;
     p.V = V;
     p.vtiles = (V + kPairV - 1) / kPairV;
-    p.parts = 8 * p.vtiles;
+    p.parts = 2 * p.vtiles;
     p.c = c;
     p.status = device_status;
     p.total_items = 0;

@@ -99,9 +99,9 @@ struct LmHeadProblem {
     float* out;
     float2* partials;   // nullptr, or [rows, lmhead_parts(V)]: row-statistics partials written by the epilogue
 };
-// Number of row-statistics partials per row the projection writes: one per 32 vocabulary entries of
-// every 256-entry tile.
-inline int lmhead_parts(int V) { return 8 * ((V + 255) / 256); }
+// Number of row-statistics partials per row the projection writes: one per 128 vocabulary entries
+// (one per CTA of the pair that owns a 256-entry tile).
+inline int lmhead_parts(int V) { return 2 * ((V + 255) / 256); }
 // c = log2(e) / T, used only when partials are requested.
 cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int32_t* device_status, cudaStream_t stream);
 
