@@ -390,6 +390,10 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
     __shared__ SampleShared sh_sample;
 
     constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
+    // Launched with programmatic stream serialisation: the CTAs may be placed while the kernel before
+    // (row statistics or the LM-head projection) is still finishing; nothing it wrote is touched before
+    // this point.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // blockIdx.x = sequence * cluster size + rank in the cluster; only rank 0 writes results
     ClusterCtx cl;
     cl.size = p.cluster;
@@ -559,13 +563,15 @@ cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p_in, cudaStream_t 
     cfg.blockDim = dim3(kWalkThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = static_cast<unsigned>(p.cluster);
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(p.cluster);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // see griddepcontrol.wait in the kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     if (dt == POLYSPEC_BF16) return cudaLaunchKernelEx(&cfg, walk_kernel<POLYSPEC_BF16>, p);
     return cudaLaunchKernelEx(&cfg, walk_kernel<POLYSPEC_F32>, p);
 }
