@@ -189,7 +189,7 @@ def run_reference(args, spec):
         d = {k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}
         step = lambda: fused_oracle_time(d, n_seq, cores)[:2]
     else:
-        n_seq = min(spec.B, 8 * cores)
+        n_seq = min(spec.B, cores)          # one sequence per thread: a step of some tens of milliseconds
         sample = oracle_sample(spec, seed=args.seed, n_seq=n_seq, device=dev)
         step = lambda: oracle_time(sample, cores)
     for _ in range(args.warmup):
@@ -544,7 +544,7 @@ def run_gpu_greedy(args, spec):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="polyspec", choices=["polyspec", "reference"])
     ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
