@@ -39,9 +39,10 @@
  *     holding NaN / +inf or no finite logit) never trap: the affected sequence gets
  *     accepted_len = next_token = -1 (and -1 in every later level of a chain) and
  *     *device_status is set to POLYSPEC_ERR_BAD_INPUT_ON_DEVICE.
- *   - No kernel waits without a limit.  Should a wait on the copy engine ever run out,
- *     *device_status becomes POLYSPEC_ERR_TIMEOUT, the outputs of that call are undefined,
- *     and the kernels still return.
+ *   - No kernel polls memory without a limit.  Should a wait on a copy or on the tensor core
+ *     ever run out, *device_status becomes POLYSPEC_ERR_TIMEOUT, the outputs of that call are
+ *     undefined, and the kernels still return.  The only other waits are hardware barriers
+ *     (block, cluster, grid dependency) that every participant reaches unconditionally.
  */
 #ifndef POLYSPEC_H
 #define POLYSPEC_H
