@@ -14,11 +14,12 @@
 //     5-stage ring of (W tile, hidden half-tile) keeps about 170 KiB in flight per SM (a sixth
 //     stage measured no faster);
 //   - the accumulator lives in TMEM (lane = vocabulary entry, column = hidden row) and is
-//     read back with tcgen05.ld by four epilogue warps per CTA.
+//     read back with tcgen05.ld by eight epilogue warps per CTA.
 //
 // The grid is persistent: CTA pair i walks work items i, i + pairs, ... of a static list
 // (model, 256-entry vocabulary tile, column block), costliest model first, so the target's and
-// the drafter's projections share one launch and the tail of one fills the other's idle SMs.
+// the drafter's projections share one launch and the tail of one fills the other's idle SMs;
+// odd pairs walk their list backwards so that neighbouring pairs are in different phases.
 // Warp roles in each CTA:
 //   warp 0      TMA producer (one elected lane issues).  Both CTAs load their own tiles; all copies of a stage
 //               complete on the leader CTA's "full" barrier (no multicast anywhere)
@@ -26,7 +27,7 @@
 //               tcgen05.commit arrives on the "empty" / "accumulator full" barriers of both CTAs
 //   warps 2..9  epilogue (two warps per TMEM lane quarter, alternate 16-column chunks): TMEM ->
 //               registers -> a 2 KiB staging tile per warp -> global by 2-D TMA store; all sixteen
-//               epilogue warps of the pair arrive on the leader's "accumulator empty" barrier.
+//               epilogue warps of the pair arrive on the leader's "slot empty" barriers.
 //               On request the epilogue also emits the row statistics of the tile (the softmax
 //               normaliser partial of each hidden row over the CTA's 128 vocabulary entries, in the
 //               format of the row-statistics kernel), so the logits need no second pass for them
@@ -450,7 +451,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1) lmh
                     if (lane == 0) mbar_arrive_cluster(leader_slot_empty + 8u * slot0);
                 }
                 if (c0 + 32 < job.block_cols) tmem_ld16(t_col(c0 + 32), nxt);
-                if (v_base >= p.V || row0 + c0 >= job.rows) continue;      // nothing of this chunk exists (warp-uniform)
+                if (row0 + c0 >= job.rows) continue;                       // no such hidden rows (warp-uniform)
+                if (v_base >= p.V) {                                       // no such vocabulary entries: an empty share
+                    if (stats && lane < 16) stat_merge[quarter * kMaxCols + c0 + lane] = make_float2(kEmptyRef, 0.0f);
+                    continue;
+                }
                 // registers -> staging tile [hidden row][vocabulary entry]; one TMA store writes its 16 rows of
                 // 128 bytes, the row statistics are read from the same tile
                 if (lane == 0) tma_store_wait_read();           // the previous store has read the tile

@@ -120,6 +120,15 @@ def test_fused_reduced_size(oracle):
     assert len(set(ora["accepted_len"].tolist())) >= 3        # the draft tracks the target: several accepted lengths
 
 
+def test_fused_ragged_vocabulary(oracle):
+    """V = 5 * 256 + 40: in the last tile one CTA of the pair sees 40 entries (two of its four lane quarters none),
+    the other CTA none at all; their shares of the row statistics must come out empty, not stale."""
+    spec = synth.FusedSpec(B=6, k=3, V=1320, d_p=128, d_q=64)
+    for seed in (7, 8):                      # a second call reuses whatever the first left in shared memory
+        d = synth.make_fused(spec, seed=seed, device=DEV)
+        _fused_compare(oracle, d, lambda dl: 4 * dl / spec.temperature)
+
+
 def test_fused_config4_full(oracle):
     spec = synth.FusedSpec()
     d = synth.make_fused(spec, seed=0, device=DEV)
