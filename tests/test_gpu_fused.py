@@ -129,6 +129,13 @@ def test_fused_ragged_vocabulary(oracle):
         _fused_compare(oracle, d, lambda dl: 4 * dl / spec.temperature)
 
 
+def test_fused_more_rows_than_one_column_block(oracle):
+    """B (k + 1) = 360 hidden rows: two 256-column blocks per vocabulary tile, two alternating accumulators."""
+    spec = synth.FusedSpec(B=40, k=8, V=2048, d_p=256, d_q=128)
+    d = synth.make_fused(spec, seed=9, device=DEV)
+    _fused_compare(oracle, d, lambda dl: 4 * dl / spec.temperature)
+
+
 def test_fused_config4_full(oracle):
     spec = synth.FusedSpec()
     d = synth.make_fused(spec, seed=0, device=DEV)
