@@ -551,12 +551,16 @@ def main():
     ap.add_argument("--sigma", type=float, default=1.0, help="inter-level noise of cfg5")
     ap.add_argument("--rule", default="sampling", choices=["sampling", "greedy"],
                     help="verification rule; greedy matching is timed on the logits-path workloads only")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the batch of a logits-path workload (e.g. 512 stacked instances of the batch-1 configs)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     spec = synth.FusedSpec() if args.workload == "cfg4" else chain_spec(args.workload, args.sigma)
+    if args.batch > 0 and args.workload != "cfg4":
+        spec = synth.scaled(spec, B=args.batch)
     if args.impl == "reference":
         run_reference(args, spec)
     elif args.rule == "greedy" and args.workload != "cfg4":
