@@ -172,7 +172,7 @@ polyspec_status polyspec_verify_chain_host(
  * fp32 accumulation on the tensor cores; logits are never passed in.
  *
  *   hidden_p [B, k+1, d_p] bf16, W_p [V, d_p] bf16 (row-major, d contiguous)
- *   hidden_q [B, rows_q, d_q] bf16 with rows_q >= k (rows past k-1 are ignored), W_q [V, d_q] bf16
+ *   hidden_q [B, rows_q, d_q] bf16 with rows_q = k or k + 1 (a row k is projected but not used), W_q [V, d_q] bf16
  *   d_p, d_q multiples of 64; V a multiple of 8; all four buffers 16-byte aligned
  *   the remaining arguments are those of polyspec_verify_level
  */

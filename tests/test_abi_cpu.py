@@ -83,6 +83,77 @@ def test_calls_reject_bad_arguments_without_launching(lib):
     assert st == binding.ERR_UNSUPPORTED                # d_q not a multiple of 64
 
 
+def test_greedy_fused_and_projection_calls_reject_bad_arguments_without_launching(lib):
+    null = None
+    fake = 0x1000
+    k = (ctypes.c_int * 2)(4, 6)
+    rows = (ctypes.c_int * 3)(5, 7, 6)
+    n = ctypes.c_size_t(0)
+    assert lib.polyspec_verify_chain_greedy_workspace(3, k, rows, 8, 32000, binding.BF16, ctypes.byref(n)) == binding.OK
+    assert n.value % 256 == 0 and n.value > 0
+    assert lib.polyspec_verify_chain_greedy_workspace(3, k, rows, 8, 32000, binding.BF16, null) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_verify_chain_greedy_workspace(1, k, rows, 8, 32000, binding.BF16, ctypes.byref(n)) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_verify_chain_greedy_workspace(3, k, rows, 8, 32004, binding.BF16, ctypes.byref(n)) == binding.ERR_UNSUPPORTED
+    models = (binding.ModelLogits * 3)(binding.ModelLogits(fake, 5), binding.ModelLogits(fake, 7), binding.ModelLogits(null, 6))
+    # the drafter's logits may be NULL under greedy matching; a verifier's may not
+    st = lib.polyspec_verify_chain_greedy(models, 3, k, fake, 8, 32000, binding.BF16, fake, fake, fake, fake, null, fake, 8, null)
+    assert st == binding.ERR_WORKSPACE
+    models[1].logits = null
+    st = lib.polyspec_verify_chain_greedy(models, 3, k, fake, 8, 32000, binding.BF16, fake, fake, fake, fake, null, fake, 1 << 30, null)
+    assert st == binding.ERR_INVALID_ARG
+    models[1].logits = fake
+    st = lib.polyspec_verify_chain_greedy(models, 3, k, null, 8, 32000, binding.BF16, fake, fake, fake, fake, null, fake, 1 << 30, null)
+    assert st == binding.ERR_INVALID_ARG                # no draft tokens
+    st = lib.polyspec_verify_chain_greedy(models, 3, k, fake, 8, 32000, binding.BF16, fake, fake, fake, fake, null, fake + 16, 1 << 30, null)
+    assert st == binding.ERR_INVALID_ARG                # workspace not 256-byte aligned
+
+    # the projection alone
+    assert lib.polyspec_lm_head(null, fake, 8, 32000, 4096, fake, null, null) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_lm_head(fake, fake, 0, 32000, 4096, fake, null, null) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_lm_head(fake + 8, fake, 8, 32000, 4096, fake, null, null) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_lm_head(fake, fake, 8, 32000, 4100, fake, null, null) == binding.ERR_UNSUPPORTED
+    assert lib.polyspec_lm_head(fake, fake, 8, 32002, 4096, fake, null, null) == binding.ERR_UNSUPPORTED
+
+    # the fused call and its halves
+    f32 = ctypes.c_float
+    args = dict(B=32, k=8, V=32000, dp=4096, dq=2048)
+    assert lib.polyspec_verify_from_hidden_workspace(32, 8, 32000, 4096, 2048, ctypes.byref(n)) == binding.OK
+    need = n.value
+
+    def fused(rows_q=9, temp=1.0, ws=fake, ws_bytes=1 << 40, hp=fake, tokens=fake, nxt=fake, **kw):
+        a = dict(args, **kw)
+        return lib.polyspec_verify_from_hidden(hp, fake, fake, fake, rows_q, tokens, fake, null, a["B"], a["k"], a["V"], a["dp"], a["dq"],
+                                               f32(temp), fake, nxt, null, null, null, ws, ws_bytes, null)
+    assert fused(ws_bytes=need - 256) == binding.ERR_WORKSPACE
+    assert fused(rows_q=7) == binding.ERR_INVALID_ARG       # fewer drafter rows than the block
+    assert fused(rows_q=10) == binding.ERR_INVALID_ARG      # more than k + 1
+    assert fused(temp=0.0) == binding.ERR_INVALID_ARG
+    assert fused(hp=null) == binding.ERR_INVALID_ARG
+    assert fused(tokens=null) == binding.ERR_INVALID_ARG
+    assert fused(nxt=null) == binding.ERR_INVALID_ARG
+    assert fused(ws=null) == binding.ERR_INVALID_ARG
+    assert fused(k=33) == binding.ERR_INVALID_ARG
+    assert fused(V=32004) == binding.ERR_UNSUPPORTED
+    assert fused(dp=4100) == binding.ERR_UNSUPPORTED
+    st = lib.polyspec_from_hidden_project(fake, fake, fake, fake, 9, 32, 8, 32000, 4096, 2048, f32(float("nan")), null, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG
+    st = lib.polyspec_from_hidden_verify(9, fake, null, null, 32, 8, 32000, 4096, 2048, f32(1.0), fake, fake, null, null, null,
+                                         fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # no uniforms
+
+    # the host-buffer chain call
+    hk = (ctypes.c_int * 1)(4)
+    hrows = (ctypes.c_int * 2)(5, 4)
+    assert lib.polyspec_verify_chain_host_workspace(2, hk, hrows, 4, 32000, binding.F32, ctypes.byref(n)) == binding.OK
+    hm = (binding.ModelLogits * 2)(binding.ModelLogits(fake, 5), binding.ModelLogits(fake, 4))
+    st = lib.polyspec_verify_chain_host(hm, 2, hk, fake, fake, 4, 32000, binding.F32, f32(1.0), fake, fake, fake, fake, null,
+                                        fake, n.value - 256, null)
+    assert st == binding.ERR_WORKSPACE
+    st = lib.polyspec_verify_chain_host(hm, 2, hk, null, fake, 4, 32000, binding.F32, f32(1.0), fake, fake, fake, fake, null,
+                                        fake, n.value, null)
+    assert st == binding.ERR_INVALID_ARG
+
+
 def test_binding_raises_when_the_library_is_missing(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libpolyspec.so")

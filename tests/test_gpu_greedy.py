@@ -122,3 +122,23 @@ def test_chain_greedy_config5_full_size(oracle):
         for b in range(spec.B):
             assert (got["out_tokens"][l, b, :n[b]] == top[b, :n[b]]).all(), (l, b)
     assert got["device_status"][0] == 0
+
+
+@pytest.mark.parametrize("sigma", [0.25, 2.0])
+def test_greedy_acceptance_statistics_follow_the_closed_form(sigma):
+    """Drafts sampled from the drafter's softmax: a position matches with probability
+    gamma_j = q_j(arg max p_j), independently, so E[a] = sum_j prod_{i<=j} gamma_i and
+    E[a^2] = sum_j (2j - 1) prod_{i<=j} gamma_i at the bottom level; checked over the whole batch."""
+    spec = synth.config("cfg5", sigma=sigma)
+    d = synth.make_chain(spec, seed=41, device=DEV)
+    got = _run(d["models"], d["k"], d["draft_tokens"])
+    kb = spec.k[2]
+    top = d["models"][2][:, :kb].float().argmax(-1, keepdim=True)
+    Q = torch.softmax(d["models"][3].double() / spec.temperature, dim=-1)
+    surv = torch.cumprod(Q.gather(-1, top).squeeze(-1), dim=1)
+    j = torch.arange(1, kb + 1, device=surv.device, dtype=torch.float64)
+    a = got["accepted_len"][2].astype(np.float64)
+    for moment, expect in ((a, surv.sum(1)), (a * a, ((2 * j - 1) * surv).sum(1))):
+        diff = moment - expect.cpu().numpy()
+        se = diff.std(ddof=1) / np.sqrt(len(diff))
+        assert abs(diff.mean()) < 3.5 * se + 1e-9, (sigma, diff.mean(), se)

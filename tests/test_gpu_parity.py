@@ -229,6 +229,12 @@ def test_config5_full_size_sampled_sequences(oracle, sigma):
     diff = out["accepted_len"][2] - expect
     se = diff.std(ddof=1) / np.sqrt(len(diff))
     assert abs(diff.mean()) < 3 * se + 1e-9, (sigma, diff.mean(), se)
+    # ... and its second moment, E[a^2] = sum_j (2j - 1) P(a >= j), which fixes the variance of the acceptance length
+    j = torch.arange(1, k[2] + 1, device=alpha.device, dtype=torch.float64)
+    expect2 = ((2 * j - 1) * torch.cumprod(alpha, dim=1)).sum(1).cpu().numpy()
+    diff2 = out["accepted_len"][2].astype(np.float64) ** 2 - expect2
+    se2 = diff2.std(ddof=1) / np.sqrt(len(diff2))
+    assert abs(diff2.mean()) < 3 * se2 + 1e-9, (sigma, diff2.mean(), se2)
 
 
 def test_chain_host_entry_point_matches_device_entry_point():
