@@ -56,6 +56,25 @@ def read_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def copy_probe_gbs(dev, nbytes=1 << 30, iters=20):
+    """Device-to-device copy bandwidth of the GPU this run landed on (bytes read + bytes written per second).
+
+    Context for the roofline fraction only: boxes of one pool differ by several per cent, and the stored
+    peak was measured on one of them.  Taken outside the timed region."""
+    src = torch.empty(nbytes, dtype=torch.uint8, device=dev).fill_(1)
+    dst = torch.empty_like(src)
+    for _ in range(3):
+        dst.copy_(src)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(iters):
+        dst.copy_(src)
+    e1.record()
+    torch.cuda.synchronize()
+    return 2.0 * nbytes * iters / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -333,6 +352,7 @@ def run_gpu(args, spec):
         ms_per_step = elapsed_ms / args.steps
         value = tokens_all * args.steps / (elapsed_ms * 1e-3)
         achieved = logits_bytes / (stats_ms * 1e-3) / 1e9
+        live_copy = copy_probe_gbs(dev)
         traffic = None if STATS_TRAFFIC_PER_LOGIT_BYTE is None else STATS_TRAFFIC_PER_LOGIT_BYTE * logits_bytes
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -350,7 +370,8 @@ def run_gpu(args, spec):
             "roofline": {"bound": "hbm", "kernel": "stats_kernel (row statistics, every logit once)",
                          "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                          "traffic": traffic, "peak_source": f"of {peaks['source']}",
-                         "frac_of_nominal_8TBs": achieved / 8000.0},
+                         "frac_of_nominal_8TBs": achieved / 8000.0,
+                         "this_gpu_copy_gbs": live_copy, "frac_of_this_gpu_copy": achieved / live_copy},
             "e2e": {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
                     "matches_device_path": same},
