@@ -235,6 +235,48 @@ polyspec_status polyspec_lm_head(const void* hidden, const void* W, int rows, in
                                  int32_t* device_status, void* cuda_stream);
 
 /*
+ * polyspec_verify_level with the vocabulary sharded over n_ranks ranks (the layout a tensor-parallel
+ * LM head leaves the logits in): rank r holds entries [r * V_local, (r + 1) * V_local) of every row,
+ * as logits_p [B, k+1, V_local] and logits_q [B, k, V_local]; the rule is Algorithm 1's Verify loop
+ * and replacement / bonus token over the whole vocabulary V = n_ranks * V_local, unchanged.
+ * The normaliser, the accept tests and the inverse-CDF search need sums over all slices, so a level
+ * is three calls per rank with two small exchanges and one reduction between them, which the caller
+ * performs (all-gather, all-gather, max); the library itself never talks to another rank:
+ *
+ *   polyspec_sharded_level_stats   writes this rank's stats record (stats_record_bytes)
+ *        -- all-gather the records into [n_ranks][stats_record_bytes], rank order --
+ *   polyspec_sharded_level_decide  accept tests on every rank (identical results): accepted_len [B];
+ *                                  writes this rank's mass record (mass_record_bytes)
+ *        -- all-gather the mass records into [n_ranks][mass_record_bytes] --
+ *   polyspec_sharded_level_pick    next_token [B]: the token (index in the whole vocabulary) on the one
+ *                                  rank whose slice contains it, -1 on the others
+ *        -- max over ranks of next_token --
+ *
+ *   draft_tokens [B, k] hold indices in the whole vocabulary; uniforms, block_len, accepted_len,
+ *   p_at_draft, q_at_draft, temperature and device_status are those of polyspec_verify_level and must be
+ *   the same on every rank.  The three calls of a level share one workspace, whose contents carry from
+ *   call to call; records are opaque, 16-byte aligned device buffers.  V_local a multiple of 8,
+ *   n_ranks <= 64.  An unusable input gives accepted_len = next_token = -1 on every rank.
+ *   With n_ranks = 1 the result is bit-identical to polyspec_verify_level.
+ */
+polyspec_status polyspec_sharded_level_sizes(int B, int k, int V_local, polyspec_dtype dt, int n_ranks,
+                                             size_t* workspace_bytes, size_t* stats_record_bytes,
+                                             size_t* mass_record_bytes /* host out, all three */);
+polyspec_status polyspec_sharded_level_stats(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, int B, int k, int V_local, int rank, int n_ranks,
+    polyspec_dtype dt, float temperature, void* stats_record /* out */, int32_t* device_status,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+polyspec_status polyspec_sharded_level_decide(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms, const int32_t* block_len,
+    int B, int k, int V_local, int rank, int n_ranks, polyspec_dtype dt, float temperature,
+    const void* stats_records /* all ranks' */, int32_t* accepted_len, float* p_at_draft, float* q_at_draft,
+    void* mass_record /* out */, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+polyspec_status polyspec_sharded_level_pick(
+    const void* logits_p, const void* logits_q, const float* uniforms, int B, int k, int V_local, int rank, int n_ranks,
+    polyspec_dtype dt, float temperature, const void* mass_records /* all ranks' */, int32_t* next_token,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Cost model of Section 3.2 (host arithmetic only; nothing is launched).
  *
  * polyspec_cost_total_time -- Lemma 3.1 (Eq. 3): the time to generate N tokens with n models,

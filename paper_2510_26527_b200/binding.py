@@ -32,6 +32,8 @@ EXPORTS = (
     "polyspec_from_hidden_project", "polyspec_from_hidden_verify",
     "polyspec_static_scratch_bytes", "polyspec_verify_level_static",
     "polyspec_cost_total_time", "polyspec_cost_insertion",
+    "polyspec_sharded_level_sizes", "polyspec_sharded_level_stats", "polyspec_sharded_level_decide",
+    "polyspec_sharded_level_pick",
 )
 
 
@@ -113,6 +115,15 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_verify_level_static.restype = ci
     lib.polyspec_verify_level_static.argtypes = [vp, vp, i32p, f32p, i32p, ci, ci, ci, ci, cf,
                                                  i32p, i32p, f32p, f32p, i32p, vp]
+    lib.polyspec_sharded_level_sizes.restype = ci
+    lib.polyspec_sharded_level_sizes.argtypes = [ci, ci, ci, ci, ci, szp, szp, szp]
+    lib.polyspec_sharded_level_stats.restype = ci
+    lib.polyspec_sharded_level_stats.argtypes = [vp, vp, i32p, ci, ci, ci, ci, ci, ci, cf, vp, i32p, vp, sz, vp]
+    lib.polyspec_sharded_level_decide.restype = ci
+    lib.polyspec_sharded_level_decide.argtypes = [vp, vp, i32p, f32p, i32p, ci, ci, ci, ci, ci, ci, cf, vp,
+                                                  i32p, f32p, f32p, vp, i32p, vp, sz, vp]
+    lib.polyspec_sharded_level_pick.restype = ci
+    lib.polyspec_sharded_level_pick.argtypes = [vp, vp, f32p, ci, ci, ci, ci, ci, ci, cf, vp, i32p, i32p, vp, sz, vp]
     _lib = lib
     return lib
 
@@ -544,3 +555,75 @@ def polyspec_cost_insertion(T_new: float, T_i: float, L_new: float, L_i: float, 
     if r < 0:
         raise ValueError("all five quantities must be positive")
     return bool(r), lhs.value, rhs.value
+
+
+# ------------------------------------------------------------------ one level, vocabulary sharded over ranks
+def polyspec_sharded_level_sizes(B: int, k: int, V_local: int, dt: int, n_ranks: int):
+    """(workspace bytes, stats record bytes, mass record bytes) of the sharded level calls."""
+    w, a, m = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(load_library().polyspec_sharded_level_sizes(B, k, V_local, dt, n_ranks, ctypes.byref(w), ctypes.byref(a), ctypes.byref(m)),
+           "polyspec_sharded_level_sizes")
+    return w.value, a.value, m.value
+
+
+class ShardedLevelCall:
+    """One rank's side of a vocabulary-sharded level: its slices of the logits, its workspace and records.
+
+    stats() -> this rank's stats record; decide(all ranks' stats records) -> (accepted_len, this rank's mass
+    record); pick(all ranks' mass records) -> next_token, -1 unless this rank's slice holds the token.  The
+    exchanges between the calls are the caller's (see paper_2510_26527_b200.sharded)."""
+
+    def __init__(self, logits_p, logits_q, draft_tokens, uniforms, temperature, rank, n_ranks, block_len=None,
+                 want_probs=False, stream=None):
+        self.lib = load_library()
+        _dev_check(logits_p, logits_q, draft_tokens, uniforms, block_len)
+        self.B, rows_p, self.V_local = logits_p.shape
+        self.k = int(draft_tokens.shape[1])
+        if rows_p != self.k + 1 or tuple(logits_q.shape) != (self.B, self.k, self.V_local) or logits_q.dtype != logits_p.dtype:
+            raise ValueError("shapes must be logits_p [B,k+1,V_local], logits_q [B,k,V_local] of one dtype")
+        self.dt = _dt(logits_p)
+        self.t = (logits_p, logits_q, draft_tokens, uniforms, block_len)
+        self.rank, self.n_ranks = int(rank), int(n_ranks)
+        self.temperature = float(temperature)
+        dev = logits_p.device
+        wbytes, self.stats_bytes, self.mass_bytes = polyspec_sharded_level_sizes(self.B, self.k, self.V_local, self.dt, self.n_ranks)
+        self.workspace = _workspace(wbytes, dev)
+        self.stats_record = torch.zeros(self.stats_bytes, dtype=torch.uint8, device=dev)
+        self.mass_record = torch.zeros(self.mass_bytes, dtype=torch.uint8, device=dev)
+        self.accepted_len = torch.empty(self.B, dtype=torch.int32, device=dev)
+        self.next_token = torch.empty(self.B, dtype=torch.int32, device=dev)
+        self.p_at = torch.zeros((self.B, self.k), dtype=torch.float32, device=dev) if want_probs else None
+        self.q_at = torch.zeros((self.B, self.k), dtype=torch.float32, device=dev) if want_probs else None
+        self.device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.stream = stream
+
+    def _sizes(self):
+        return (self.B, self.k, self.V_local, self.rank, self.n_ranks, self.dt, self.temperature)
+
+    def _tail(self):
+        return (_ptr(self.device_status), _ptr(self.workspace), self.workspace.numel(), _stream(self.stream))
+
+    def stats(self):
+        lp, lq, tok, _, _ = self.t
+        _check(self.lib.polyspec_sharded_level_stats(_ptr(lp), _ptr(lq), _ptr(tok), *self._sizes(), _ptr(self.stats_record), *self._tail()),
+               "polyspec_sharded_level_stats")
+        return self.stats_record
+
+    def decide(self, stats_records):
+        lp, lq, tok, u, bl = self.t
+        _dev_check(stats_records)
+        if stats_records.numel() != self.n_ranks * self.stats_bytes:
+            raise ValueError("need every rank's stats record, in rank order")
+        _check(self.lib.polyspec_sharded_level_decide(_ptr(lp), _ptr(lq), _ptr(tok), _ptr(u), _ptr(bl), *self._sizes(), _ptr(stats_records),
+                                                      _ptr(self.accepted_len), _ptr(self.p_at), _ptr(self.q_at), _ptr(self.mass_record),
+                                                      *self._tail()), "polyspec_sharded_level_decide")
+        return self.accepted_len, self.mass_record
+
+    def pick(self, mass_records):
+        lp, lq, _, u, _ = self.t
+        _dev_check(mass_records)
+        if mass_records.numel() != self.n_ranks * self.mass_bytes:
+            raise ValueError("need every rank's mass record, in rank order")
+        _check(self.lib.polyspec_sharded_level_pick(_ptr(lp), _ptr(lq), _ptr(u), *self._sizes(), _ptr(mass_records), _ptr(self.next_token),
+                                                    *self._tail()), "polyspec_sharded_level_pick")
+        return self.next_token

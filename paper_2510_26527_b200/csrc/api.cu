@@ -13,12 +13,6 @@ constexpr double kLog2e = 1.4426950408889634074;
 
 // The runtime's code for the most recent POLYSPEC_ERR_CUDA (see polyspec_last_cuda_error).
 cudaError_t g_last_cuda_error = cudaSuccess;
-inline bool cuda_failed(cudaError_t e)
-{
-    if (e == cudaSuccess) return false;
-    g_last_cuda_error = e;
-    return true;
-}
 
 inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -183,6 +177,13 @@ ChainArgs chain_args(const polyspec_model_logits* models, int n_models, const in
 }
 
 }  // namespace
+
+bool polyspec::cuda_failed(cudaError_t e)
+{
+    if (e == cudaSuccess) return false;
+    g_last_cuda_error = e;
+    return true;
+}
 
 extern "C" {
 

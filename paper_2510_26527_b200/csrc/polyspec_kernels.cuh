@@ -13,6 +13,9 @@ constexpr int kMaxModels = POLYSPEC_MAX_MODELS;
 constexpr int kMaxLevels = POLYSPEC_MAX_MODELS - 1;
 constexpr int kMaxK = POLYSPEC_MAX_K;
 
+// Records the runtime's code for polyspec_last_cuda_error; true if `e` is an error.
+bool cuda_failed(cudaError_t e);
+
 // Reference exponent of a stretch of a row that holds no finite logit (its sum is 0).
 constexpr float kEmptyRef = -1.0e30f;
 

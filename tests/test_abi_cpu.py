@@ -154,6 +154,38 @@ def test_greedy_fused_and_projection_calls_reject_bad_arguments_without_launchin
     assert st == binding.ERR_INVALID_ARG
 
 
+def test_sharded_level_calls_reject_bad_arguments_without_launching(lib):
+    null, fake = None, 0x1000
+    f32 = ctypes.c_float
+    w, a, m = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_size_t(0)
+    ok = lib.polyspec_sharded_level_sizes(64, 6, 16032, binding.BF16, 8, ctypes.byref(w), ctypes.byref(a), ctypes.byref(m))
+    assert ok == binding.OK
+    assert w.value % 256 == 0 and a.value >= 64 * (13 * 12 + 12 * 4) and m.value >= 64 * 16
+    for args, st in (((0, 6, 16032, binding.BF16, 8), binding.ERR_INVALID_ARG),
+                     ((64, 33, 16032, binding.BF16, 8), binding.ERR_INVALID_ARG),
+                     ((64, 6, 16032, binding.BF16, 0), binding.ERR_INVALID_ARG),
+                     ((64, 6, 16032, binding.BF16, 65), binding.ERR_INVALID_ARG),
+                     ((64, 6, 16036, binding.BF16, 8), binding.ERR_UNSUPPORTED),        # slice not a multiple of 8
+                     ((64, 6, 1 << 21, binding.BF16, 2048 // 64 * 64), binding.ERR_INVALID_ARG)):
+        assert lib.polyspec_sharded_level_sizes(*args, ctypes.byref(w), ctypes.byref(a), ctypes.byref(m)) == st, args
+    assert lib.polyspec_sharded_level_sizes(64, 6, 16032, binding.BF16, 8, null, ctypes.byref(a), ctypes.byref(m)) == binding.ERR_INVALID_ARG
+    lib.polyspec_sharded_level_sizes(64, 6, 16032, binding.BF16, 8, ctypes.byref(w), ctypes.byref(a), ctypes.byref(m))
+
+    def stats(rank=0, ws_bytes=1 << 40, rec=fake, temp=1.0, lp=fake):
+        return lib.polyspec_sharded_level_stats(lp, fake, fake, 64, 6, 16032, rank, 8, binding.BF16, f32(temp), rec, null, fake, ws_bytes, null)
+    assert stats(rank=8) == binding.ERR_INVALID_ARG
+    assert stats(rank=-1) == binding.ERR_INVALID_ARG
+    assert stats(ws_bytes=w.value - 256) == binding.ERR_WORKSPACE
+    assert stats(rec=null) == binding.ERR_INVALID_ARG
+    assert stats(temp=0.0) == binding.ERR_INVALID_ARG
+    assert stats(lp=fake + 8) == binding.ERR_INVALID_ARG
+    st = lib.polyspec_sharded_level_decide(fake, fake, fake, fake, null, 64, 6, 16032, 0, 8, binding.BF16, f32(1.0), null,
+                                           fake, null, null, fake, null, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # no stats records
+    st = lib.polyspec_sharded_level_pick(fake, fake, fake, 64, 6, 16032, 0, 8, binding.BF16, f32(1.0), fake, null, null, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # nowhere to put the token
+
+
 def test_binding_raises_when_the_library_is_missing(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libpolyspec.so")
