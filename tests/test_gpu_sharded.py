@@ -75,6 +75,27 @@ def test_several_ranks_against_the_oracle(oracle, dtype, R, V, k):
     assert same.sum() >= B - 2
 
 
+def test_full_size_level_eight_ranks(oracle):
+    """The bottom level of the four-model workload at full size (B=256, k=10, V=152064, bf16) over eight ranks:
+    sampled sequences against the oracle, the whole batch against the unsharded call."""
+    spec = synth.config("cfg5", sigma=1.0)
+    d = synth.make_chain(spec, seed=7, device=DEV)
+    lp, lq = d["models"][2].contiguous(), d["models"][3].contiguous()
+    tok, u, T = d["draft_tokens"], d["uniforms"][2].contiguous(), spec.temperature
+    del d
+    a, t, status, _ = _run_sharded(lp, lq, tok, u, T, 8)
+    assert status == 0
+    seqs = [0, 1, 2, 100, 101, 253, 254, 255]
+    ora = oracle.verify_level(lp[seqs].cpu(), lq[seqs].cpu(), tok[seqs].cpu(), u[seqs].cpu(), T, threads=8)
+    counts, bad = H.compare_level_batch(a[seqs], t[seqs], ora)
+    assert not bad, bad[:5]
+    want = binding.polyspec_verify_level(lp, lq, tok, u, T)
+    torch.cuda.synchronize()
+    same = (a == want["accepted_len"].cpu().numpy()) & (t == want["next_token"].cpu().numpy())
+    assert same.sum() >= len(a) - 2
+    assert (t >= 0).all() and (t < spec.V).all()
+
+
 def test_block_len_identical_models_and_probabilities(oracle):
     B, k, V, R = 66, 5, 2048, 4
     g = torch.Generator(device=DEV).manual_seed(1)
