@@ -202,7 +202,7 @@ const char* polyspec_status_string(polyspec_status s)
     return "unknown status";
 }
 
-int polyspec_version(void) { return 100; }
+int polyspec_version(void) { return 200; }      // 0.2.0: greedy matching, cost model, sharded level added to the ABI
 
 const char* polyspec_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
