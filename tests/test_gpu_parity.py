@@ -332,3 +332,40 @@ def test_halves_of_the_chain_call_equal_the_whole_call():
     again = _np(call.launch())
     for key in ("accepted_len", "block_len", "out_tokens", "out_len"):
         assert (again[key] == whole[key]).all()
+
+
+@pytest.mark.parametrize("n_models", [2, 3, 4])
+def test_committed_tokens_follow_the_target_distribution(n_models):
+    """Losslessness, measured on the GPU without the oracle: whatever the drafters are, the first committed token
+    is a sample of the target's first row and, given that it was accepted, so is the second of its second row
+    (Section 3.1: the verification rule preserves the target distribution).  Every sequence sees the same logits,
+    the drafts are drawn from the bottom drafter per sequence and the uniforms are Philox draws, so the committed
+    tokens are i.i.d.; chi-square against the float64 softmax."""
+    from scipy import stats as sps
+    B, V, T = 300_000, 48, 0.8
+    k = [3, 4, 5][: n_models - 1]
+    g = torch.Generator(device=DEV).manual_seed(11 + n_models)
+    rows = [k[l] + 1 for l in range(n_models - 1)] + [k[-1]]
+    base = torch.randn((max(rows), V), generator=g, device=DEV) * 2.0
+    models = []
+    for i in range(n_models):
+        one = base[: rows[i]] + (0.8 * i) * torch.randn((rows[i], V), generator=g, device=DEV)
+        models.append(one.unsqueeze(0).expand(B, rows[i], V).contiguous())
+    q = torch.softmax(models[-1][0].double() / T, dim=-1)
+    draft = torch.multinomial(q, B, replacement=True, generator=g).t().contiguous().to(torch.int32)      # [B, k_bottom]
+    u = torch.from_numpy(synth.philox_uniforms(77, n_models - 1, B, max(k) + 1)).to(DEV)
+    out = _np(binding.polyspec_verify_chain(models, k, draft, u, T))
+    assert out["device_status"][0] == 0
+    p0 = torch.softmax(models[0][0, 0].double() / T, dim=-1).cpu().numpy()
+    first = out["out_tokens"][0, :, 0]
+    counts = np.bincount(first, minlength=V).astype(np.float64)
+    chi2 = ((counts - B * p0) ** 2 / (B * p0)).sum()
+    assert chi2 < sps.chi2.ppf(1 - 1e-6, V - 1), (n_models, chi2)
+    # second committed token, for the sequences that committed at least two: a sample of row 1
+    two = out["out_len"][0] >= 2
+    p1 = torch.softmax(models[0][0, 1].double() / T, dim=-1).cpu().numpy()
+    c1 = np.bincount(out["out_tokens"][0, two, 1], minlength=V).astype(np.float64)
+    n1 = two.sum()
+    assert n1 > B // 20
+    chi2 = ((c1 - n1 * p1) ** 2 / (n1 * p1)).sum()
+    assert chi2 < sps.chi2.ppf(1 - 1e-6, V - 1), (n_models, "second", chi2)
