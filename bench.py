@@ -344,7 +344,7 @@ def run_gpu(args, spec):
         [elapsed_ms, e2e_ms, stats_ms, walk_ms], [tokens_per_step, emitted_per_step], dev, world)
 
     base = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:      # the CPU baseline is a one-GPU-run extra
         base = cpu_baseline(data, spec, target_seconds=args.cpu_seconds)
 
     if rank == 0:
@@ -469,7 +469,7 @@ def run_gpu_fused(args, spec):
         [elapsed_ms, e2e_ms, gemm_ms, verify_ms], [tokens_per_step, emitted_per_step], dev, world)
 
     base = None
-    if rank == 0 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:      # the CPU baseline is a one-GPU-run extra
         base = fused_cpu_baseline({k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}, spec, target_seconds=args.cpu_seconds)
 
     if rank == 0:
