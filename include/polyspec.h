@@ -277,6 +277,49 @@ polyspec_status polyspec_sharded_level_pick(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * polyspec_verify_chain with the vocabulary sharded over n_ranks ranks: every model's logits as
+ * [B, rows, V_local] slices (models[i].logits, models[i].rows as in polyspec_verify_chain), levels verified
+ * bottom-up (Section 3.1).  One stats call covers every row of every model; each level then takes a
+ * gather call (the logits at its block tokens, which only exist once the level below is done), decide
+ * and pick as in the single-level calls, and a hand-off that turns (accepted length, token) into the
+ * block of the level above.  Per chain: all-gather of the stats records; per level, for
+ * level = n_models-2 down to 0: all-gather of the gather records, all-gather of the mass records, max of
+ * next_token, then polyspec_sharded_chain_handoff on every rank.
+ *
+ *   block_tokens [B, kmax+1], block_len [B]: the block the current level verifies, the same on every
+ *       rank; the caller fills them with the draft tokens and k[n_models-2] (or fewer) before the
+ *       bottom level, the hand-off rewrites them for the level above (block_len -1: unusable input below)
+ *   uniforms [n_models-1, B, kmax+1], accepted_len, block_len_out, out_tokens, out_len: those of
+ *       polyspec_verify_chain (block_len_out is its block_len output); each call touches its level's part
+ *   With n_ranks = 1 the four outputs are bit-identical to polyspec_verify_chain's.
+ */
+polyspec_status polyspec_sharded_chain_sizes(int n_models, const int* k /* host */, const int* rows /* host [n_models] */, int B,
+                                             int V_local, polyspec_dtype dt, int n_ranks, size_t* workspace_bytes,
+                                             size_t* stats_record_bytes, size_t* gather_record_bytes,
+                                             size_t* mass_record_bytes /* host out, all four */);
+polyspec_status polyspec_sharded_chain_stats(
+    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */, int B, int V_local, int rank, int n_ranks,
+    polyspec_dtype dt, float temperature, void* stats_record /* out */, int32_t* device_status,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+polyspec_status polyspec_sharded_chain_gather(
+    const polyspec_model_logits* models, int n_models, const int* k, int level, const int32_t* block_tokens, const int32_t* block_len,
+    int B, int V_local, int rank, int n_ranks, polyspec_dtype dt, void* gather_record /* out */,
+    void* workspace, size_t workspace_bytes, void* cuda_stream);
+polyspec_status polyspec_sharded_chain_decide(
+    const polyspec_model_logits* models, int n_models, const int* k, int level, const int32_t* block_tokens, const int32_t* block_len,
+    const float* uniforms, int B, int V_local, int rank, int n_ranks, polyspec_dtype dt, float temperature,
+    const void* stats_records /* all ranks' */, const void* gather_records /* all ranks' */, int32_t* accepted_len,
+    int32_t* block_len_out, void* mass_record /* out */, int32_t* device_status, void* workspace, size_t workspace_bytes,
+    void* cuda_stream);
+polyspec_status polyspec_sharded_chain_pick(
+    const polyspec_model_logits* models, int n_models, const int* k, int level, const float* uniforms, int B, int V_local, int rank,
+    int n_ranks, polyspec_dtype dt, float temperature, const void* mass_records /* all ranks' */, int32_t* next_token /* [B] */,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
+polyspec_status polyspec_sharded_chain_handoff(
+    int n_models, const int* k, int level, int B, const int32_t* accepted_len, const int32_t* next_token /* after the max */,
+    int32_t* block_tokens /* in/out */, int32_t* block_len /* in/out */, int32_t* out_tokens, int32_t* out_len, void* cuda_stream);
+
+/*
  * Cost model of Section 3.2 (host arithmetic only; nothing is launched).
  *
  * polyspec_cost_total_time -- Lemma 3.1 (Eq. 3): the time to generate N tokens with n models,

@@ -34,6 +34,8 @@ EXPORTS = (
     "polyspec_cost_total_time", "polyspec_cost_insertion",
     "polyspec_sharded_level_sizes", "polyspec_sharded_level_stats", "polyspec_sharded_level_decide",
     "polyspec_sharded_level_pick",
+    "polyspec_sharded_chain_sizes", "polyspec_sharded_chain_stats", "polyspec_sharded_chain_gather",
+    "polyspec_sharded_chain_decide", "polyspec_sharded_chain_pick", "polyspec_sharded_chain_handoff",
 )
 
 
@@ -124,6 +126,20 @@ def load_library() -> ctypes.CDLL:
                                                   i32p, f32p, f32p, vp, i32p, vp, sz, vp]
     lib.polyspec_sharded_level_pick.restype = ci
     lib.polyspec_sharded_level_pick.argtypes = [vp, vp, f32p, ci, ci, ci, ci, ci, ci, cf, vp, i32p, i32p, vp, sz, vp]
+    mlp = ctypes.POINTER(ModelLogits)
+    lib.polyspec_sharded_chain_sizes.restype = ci
+    lib.polyspec_sharded_chain_sizes.argtypes = [ci, cip, cip, ci, ci, ci, ci, szp, szp, szp, szp]
+    lib.polyspec_sharded_chain_stats.restype = ci
+    lib.polyspec_sharded_chain_stats.argtypes = [mlp, ci, cip, ci, ci, ci, ci, ci, cf, vp, i32p, vp, sz, vp]
+    lib.polyspec_sharded_chain_gather.restype = ci
+    lib.polyspec_sharded_chain_gather.argtypes = [mlp, ci, cip, ci, i32p, i32p, ci, ci, ci, ci, ci, vp, vp, sz, vp]
+    lib.polyspec_sharded_chain_decide.restype = ci
+    lib.polyspec_sharded_chain_decide.argtypes = [mlp, ci, cip, ci, i32p, i32p, f32p, ci, ci, ci, ci, ci, cf, vp, vp, i32p, i32p, vp,
+                                                  i32p, vp, sz, vp]
+    lib.polyspec_sharded_chain_pick.restype = ci
+    lib.polyspec_sharded_chain_pick.argtypes = [mlp, ci, cip, ci, f32p, ci, ci, ci, ci, ci, cf, vp, i32p, i32p, vp, sz, vp]
+    lib.polyspec_sharded_chain_handoff.restype = ci
+    lib.polyspec_sharded_chain_handoff.argtypes = [ci, cip, ci, ci, i32p, i32p, i32p, i32p, i32p, i32p, vp]
     _lib = lib
     return lib
 
@@ -627,3 +643,100 @@ class ShardedLevelCall:
         _check(self.lib.polyspec_sharded_level_pick(_ptr(lp), _ptr(lq), _ptr(u), *self._sizes(), _ptr(mass_records), _ptr(self.next_token),
                                                     *self._tail()), "polyspec_sharded_level_pick")
         return self.next_token
+
+
+def polyspec_sharded_chain_sizes(k: Sequence[int], rows: Sequence[int], B: int, V_local: int, dt: int, n_ranks: int):
+    """(workspace, stats record, gather record, mass record) bytes of the sharded chain calls."""
+    w, a, g, m = (ctypes.c_size_t(0) for _ in range(4))
+    _check(load_library().polyspec_sharded_chain_sizes(len(rows), _int_array(k), _int_array(rows), B, V_local, dt, n_ranks,
+                                                       ctypes.byref(w), ctypes.byref(a), ctypes.byref(g), ctypes.byref(m)),
+           "polyspec_sharded_chain_sizes")
+    return w.value, a.value, g.value, m.value
+
+
+class ShardedChainCall:
+    """One rank's side of a vocabulary-sharded chain: its slices of every model's logits, its workspace, records,
+    the block being verified and the chain's outputs (identical on every rank once a level is handed off).
+
+    stats() once; then per level, bottom-up: gather(level), decide(level, stats records, gather records),
+    pick(level, mass records), handoff(level, token after the max over ranks)."""
+
+    def __init__(self, models, k, draft_tokens, uniforms, temperature, rank, n_ranks, stream=None):
+        self.lib = load_library()
+        _dev_check(*models, draft_tokens, uniforms)
+        self.models = list(models)
+        self.n = len(models)
+        self.L = self.n - 1
+        self.B, _, self.V_local = models[0].shape
+        self.dt = _dt(models[0])
+        self.rows = [int(m.shape[1]) for m in models]
+        self.k = [int(x) for x in k]
+        self.kmax = max(self.k)
+        if any(m.dtype != models[0].dtype or m.shape[0] != self.B or m.shape[2] != self.V_local for m in models):
+            raise ValueError("every model's slice must be [B, rows, V_local] of one dtype")
+        if tuple(draft_tokens.shape) != (self.B, self.k[-1]) or tuple(uniforms.shape) != (self.L, self.B, self.kmax + 1):
+            raise ValueError("shapes must be draft_tokens [B, k[-1]], uniforms [n_models-1, B, kmax+1]")
+        self.rank, self.n_ranks = int(rank), int(n_ranks)
+        self.temperature = float(temperature)
+        self.uniforms = uniforms
+        dev = models[0].device
+        wbytes, self.stats_bytes, self.gather_bytes, self.mass_bytes = polyspec_sharded_chain_sizes(
+            self.k, self.rows, self.B, self.V_local, self.dt, self.n_ranks)
+        self.workspace = _workspace(wbytes, dev)
+        self.stats_record = torch.zeros(self.stats_bytes, dtype=torch.uint8, device=dev)
+        self.gather_record = torch.zeros(self.gather_bytes, dtype=torch.uint8, device=dev)
+        self.mass_record = torch.zeros(self.mass_bytes, dtype=torch.uint8, device=dev)
+        self.block_tokens = torch.full((self.B, self.kmax + 1), -1, dtype=torch.int32, device=dev)
+        self.block_tokens[:, : self.k[-1]] = draft_tokens
+        self.block_len = torch.full((self.B,), self.k[-1], dtype=torch.int32, device=dev)
+        self.next_token = torch.empty(self.B, dtype=torch.int32, device=dev)
+        self.out = chain_outputs(self.L, self.B, self.kmax, dev)
+        self.device_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.out["device_status"] = self.device_status
+        self._arr = (ModelLogits * self.n)(*[ModelLogits(m.data_ptr(), r) for m, r in zip(models, self.rows)])
+        self._k = _int_array(self.k)
+        self.stream = stream
+
+    def _head(self):
+        return (self._arr, self.n, self._k)
+
+    def _geom(self):
+        return (self.B, self.V_local, self.rank, self.n_ranks, self.dt)
+
+    def _ws(self):
+        return (_ptr(self.workspace), self.workspace.numel(), _stream(self.stream))
+
+    def stats(self):
+        _check(self.lib.polyspec_sharded_chain_stats(*self._head(), *self._geom(), self.temperature, _ptr(self.stats_record),
+                                                     _ptr(self.device_status), *self._ws()), "polyspec_sharded_chain_stats")
+        return self.stats_record
+
+    def gather(self, level):
+        _check(self.lib.polyspec_sharded_chain_gather(*self._head(), level, _ptr(self.block_tokens), _ptr(self.block_len), *self._geom(),
+                                                      _ptr(self.gather_record), *self._ws()), "polyspec_sharded_chain_gather")
+        return self.gather_record
+
+    def decide(self, level, stats_records, gather_records):
+        _dev_check(stats_records, gather_records)
+        if stats_records.numel() != self.n_ranks * self.stats_bytes or gather_records.numel() != self.n_ranks * self.gather_bytes:
+            raise ValueError("need every rank's records, in rank order")
+        _check(self.lib.polyspec_sharded_chain_decide(*self._head(), level, _ptr(self.block_tokens), _ptr(self.block_len), _ptr(self.uniforms),
+                                                      *self._geom(), self.temperature, _ptr(stats_records), _ptr(gather_records),
+                                                      _ptr(self.out["accepted_len"]), _ptr(self.out["block_len"]), _ptr(self.mass_record),
+                                                      _ptr(self.device_status), *self._ws()), "polyspec_sharded_chain_decide")
+        return self.mass_record
+
+    def pick(self, level, mass_records):
+        _dev_check(mass_records)
+        if mass_records.numel() != self.n_ranks * self.mass_bytes:
+            raise ValueError("need every rank's mass record, in rank order")
+        _check(self.lib.polyspec_sharded_chain_pick(*self._head(), level, _ptr(self.uniforms), *self._geom(), self.temperature,
+                                                    _ptr(mass_records), _ptr(self.next_token), _ptr(self.device_status), *self._ws()),
+               "polyspec_sharded_chain_pick")
+        return self.next_token
+
+    def handoff(self, level, token):
+        _dev_check(token)
+        _check(self.lib.polyspec_sharded_chain_handoff(self.n, self._k, level, self.B, _ptr(self.out["accepted_len"]), _ptr(token),
+                                                       _ptr(self.block_tokens), _ptr(self.block_len), _ptr(self.out["out_tokens"]),
+                                                       _ptr(self.out["out_len"]), _stream(self.stream)), "polyspec_sharded_chain_handoff")

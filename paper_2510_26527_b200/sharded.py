@@ -53,3 +53,33 @@ def verify_level_sharded_on_one_device(calls: Sequence) -> tuple:
     masses = torch.cat([m for _, m in decided]).contiguous()
     tokens = torch.stack([c.pick(masses) for c in calls])
     return [a for a, _ in decided], tokens.max(dim=0).values
+
+
+def _drive_chain(calls, gather, reduce_max):
+    """The order of calls and exchanges of a sharded chain, for the ranks in ``calls`` (one in a distributed run,
+    all of them when one device plays every rank)."""
+    stats = gather([c.stats() for c in calls])
+    for level in reversed(range(calls[0].L)):
+        gathers = gather([c.gather(level) for c in calls])
+        masses = gather([c.decide(level, stats, gathers) for c in calls])
+        token = reduce_max([c.pick(level, masses) for c in calls])
+        for c in calls:
+            c.handoff(level, token)
+    return calls[0].out
+
+
+def verify_chain_vocab_parallel(call, group=None):
+    """The whole chain on this rank's ``call`` (a ShardedChainCall); returns its outputs, identical on every rank."""
+    import torch.distributed as dist
+
+    def reduce_max(tokens):
+        token = tokens[0].clone()
+        dist.all_reduce(token, op=dist.ReduceOp.MAX, group=group)
+        return token
+    return _drive_chain([call], lambda recs: gather_records(recs[0], group), reduce_max)
+
+
+def verify_chain_sharded_on_one_device(calls: Sequence):
+    """All ranks' chain calls on one device, phase by phase (see verify_level_sharded_on_one_device)."""
+    return _drive_chain(list(calls), lambda recs: torch.cat(list(recs)).contiguous(),
+                        lambda tokens: torch.stack(list(tokens)).max(dim=0).values.contiguous())

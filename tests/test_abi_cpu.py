@@ -186,6 +186,36 @@ def test_sharded_level_calls_reject_bad_arguments_without_launching(lib):
     assert st == binding.ERR_INVALID_ARG                # nowhere to put the token
 
 
+def test_sharded_chain_calls_reject_bad_arguments_without_launching(lib):
+    null, fake = None, 0x1000
+    f32 = ctypes.c_float
+    k = (ctypes.c_int * 3)(4, 6, 10)
+    rows = (ctypes.c_int * 4)(5, 7, 11, 10)
+    sizes = [ctypes.c_size_t(0) for _ in range(4)]
+    refs = [ctypes.byref(x) for x in sizes]
+    assert lib.polyspec_sharded_chain_sizes(4, k, rows, 256, 19008, binding.BF16, 8, *refs) == binding.OK
+    w, a, g, m = (x.value for x in sizes)
+    assert a >= 256 * 33 * 12 and g >= 256 * 11 * 8 and m >= 256 * 16 and all(x % 256 == 0 for x in (w, a, g, m))
+    assert lib.polyspec_sharded_chain_sizes(1, k, rows, 256, 19008, binding.BF16, 8, *refs) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_sharded_chain_sizes(4, k, rows, 256, 19004, binding.BF16, 8, *refs) == binding.ERR_UNSUPPORTED
+    short = (ctypes.c_int * 4)(5, 6, 11, 10)                           # model 1 lacks its bonus row
+    assert lib.polyspec_sharded_chain_sizes(4, k, short, 256, 19008, binding.BF16, 8, *refs) == binding.ERR_INVALID_ARG
+    models = (binding.ModelLogits * 4)(*[binding.ModelLogits(fake, r) for r in (5, 7, 11, 10)])
+    st = lib.polyspec_sharded_chain_stats(models, 4, k, 256, 19008, 8, 8, binding.BF16, f32(1.0), fake, null, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # rank out of range
+    st = lib.polyspec_sharded_chain_stats(models, 4, k, 256, 19008, 0, 8, binding.BF16, f32(1.0), fake, null, fake, w - 256, null)
+    assert st == binding.ERR_WORKSPACE
+    st = lib.polyspec_sharded_chain_gather(models, 4, k, 3, fake, fake, 256, 19008, 0, 8, binding.BF16, fake, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # no such level
+    st = lib.polyspec_sharded_chain_decide(models, 4, k, 2, fake, fake, fake, 256, 19008, 0, 8, binding.BF16, f32(1.0), fake, null,
+                                           fake, null, fake, null, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # no gather records
+    st = lib.polyspec_sharded_chain_pick(models, 4, k, 2, fake, 256, 19008, 0, 8, binding.BF16, f32(-1.0), fake, fake, null, fake, 1 << 40, null)
+    assert st == binding.ERR_INVALID_ARG                # temperature
+    assert lib.polyspec_sharded_chain_handoff(4, k, 3, 256, fake, fake, fake, fake, null, null, null) == binding.ERR_INVALID_ARG
+    assert lib.polyspec_sharded_chain_handoff(4, k, 0, 256, fake, null, fake, fake, null, null, null) == binding.ERR_INVALID_ARG
+
+
 def test_binding_raises_when_the_library_is_missing(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libpolyspec.so")

@@ -182,3 +182,65 @@ def test_argument_checks():
         binding.polyspec_sharded_level_sizes(2, 2, 60, binding.F32, 2)                  # slice not a multiple of 8
     with pytest.raises(binding.PolyspecError):
         binding.polyspec_sharded_level_sizes(2, 2, 64, binding.F32, 65)                 # too many ranks
+
+
+# ------------------------------------------------------------------------------------------------ chains
+CHAIN_KEYS = ("accepted_len", "block_len", "out_len", "out_tokens")
+
+
+def _run_sharded_chain(d, R):
+    shards = [sharded.shard_vocabulary(m, R) for m in d["models"]]
+    calls = [binding.ShardedChainCall([s[r] for s in shards], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"], r, R)
+             for r in range(R)]
+    out = sharded.verify_chain_sharded_on_one_device(calls)
+    torch.cuda.synchronize()
+    for c in calls[1:]:
+        for key in CHAIN_KEYS:
+            assert torch.equal(c.out[key], out[key]), key            # every rank ends with the same outputs
+    status = max(int(c.device_status[0]) for c in calls)
+    return {key: out[key].cpu().numpy() for key in CHAIN_KEYS}, status
+
+
+@pytest.mark.parametrize("name,B,V,sigma", [("cfg1", 40, 4096, None), ("cfg2", 24, 4096, None), ("cfg3", 16, 10000, None),
+                                            ("cfg5", 12, 8200, 0.5)])
+def test_chain_one_rank_is_bit_identical_to_verify_chain(name, B, V, sigma):
+    spec = synth.scaled(synth.config(name, sigma=sigma), B=B, V=V)
+    d = synth.make_chain(spec, seed=61, device=DEV)
+    want = binding.polyspec_verify_chain(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    torch.cuda.synchronize()
+    got, status = _run_sharded_chain(d, 1)
+    assert status == 0
+    for key in CHAIN_KEYS:
+        assert (got[key] == want[key].cpu().numpy()).all(), key
+
+
+@pytest.mark.parametrize("name,B,V,sigma,R", [("cfg2", 24, 4096, None, 2), ("cfg3", 16, 10240, None, 4), ("cfg5", 12, 8192, 0.5, 8),
+                                              ("cfg5", 16, 8200, 1.0, 5), ("cfg5", 8, 152064, 0.25, 8)])
+def test_chain_several_ranks_against_the_oracle(oracle, name, B, V, sigma, R):
+    spec = synth.scaled(synth.config(name, sigma=sigma), B=B, V=V)
+    d = synth.make_chain(spec, seed=62, device=DEV)
+    got, status = _run_sharded_chain(d, R)
+    assert status == 0
+    ora = oracle.verify_chain([m.cpu() for m in d["models"]], d["k"], d["draft_tokens"].cpu(), d["uniforms"].cpu(),
+                              d["temperature"], threads=8)
+    counts, bad = H.compare_chain(got, ora)
+    print(f"[parity] sharded chain {name} R={R}: {counts}")
+    assert not bad, bad[:5]
+    assert counts["tie_accept"] + counts["tie_sample"] <= 2
+    assert (got["out_len"] == got["accepted_len"] + 1).all()
+
+
+def test_chain_unusable_input_below_reports_minus_one_above():
+    spec = synth.scaled(synth.config("cfg5", sigma=0.5), B=6, V=4096)
+    d = synth.make_chain(spec, seed=63, device=DEV)
+    d["draft_tokens"][2, 0] = spec.V                       # out of range at the bottom level
+    d["models"][1][4, 0, 7] = float("nan")                 # an unusable row at level 1
+    want = binding.polyspec_verify_chain(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    torch.cuda.synchronize()
+    got, status = _run_sharded_chain(d, 4)
+    assert status == binding.ERR_BAD_INPUT_ON_DEVICE
+    assert (got["accepted_len"][:, 2] == -1).all() and (got["out_len"][:, 2] == -1).all() and (got["out_tokens"][:, 2] == -1).all()
+    assert got["accepted_len"][2, 4] >= 0 and (got["accepted_len"][:2, 4] == -1).all()
+    for key in CHAIN_KEYS:
+        w = want[key].cpu().numpy()
+        assert (got[key][:, [2, 4]] == w[:, [2, 4]]).all(), key          # the same report as the unsharded call
