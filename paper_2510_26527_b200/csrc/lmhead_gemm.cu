@@ -41,6 +41,8 @@
 // (bounded again), and the kernel still frees TMEM and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "polyspec_kernels.cuh"
 
 namespace polyspec {
@@ -542,6 +544,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+std::mutex g_init_mutex;
 EncodeTiledFn g_encode = nullptr;
 bool g_attr_set[64] = {false};
 int g_pairs[64] = {0};      // CTA pairs the device can hold at once
@@ -588,6 +591,7 @@ bool encode_map(CUtensorMap* map, const void* base, int n_rows, int d, int box_r
 cudaError_t launch_lmhead(const LmHeadProblem* probs, int n, int V, float c, int32_t* device_status, cudaStream_t stream)
 {
     if (n < 1 || n > 2) return cudaErrorInvalidValue;
+    std::lock_guard<std::mutex> lock(g_init_mutex);      // one-time set-up below; host threads may call concurrently
     cudaError_t e = get_encoder();
     if (e != cudaSuccess) return e;
     int dev = 0;
