@@ -40,7 +40,7 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-statistics kernel, from the ncu
 # capture summarised under profiles/ (bytes per logits byte processed, measured on a smaller case of
 # the same kernel and scaled by the bytes one launch processes).  None until a capture exists.
-STATS_TRAFFIC_PER_LOGIT_BYTE = 1.0139     # profiles/stats_kernel_bf16_cfg3_ncu_full.md: (328.353 + 4.562) MB moved for 328.340 MB of logits
+STATS_TRAFFIC_PER_LOGIT_BYTE = 1.0130     # profiles/stats_kernel_bf16_cfg3_ncu_full.md: (328.350 + 4.250) MB moved for 328.340 MB of logits
 # the same counters per launch of the LM-head kernel on the fused workload
 # (profiles/lmhead_kernel_cfg4_ncu.md: 402.98 MB read + 53.81 MB written)
 LMHEAD_TRAFFIC_BYTES = 456789504

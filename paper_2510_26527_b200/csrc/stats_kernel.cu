@@ -100,6 +100,21 @@ template <> struct Elems<POLYSPEC_BF16> {
         z[6] = __uint_as_float(r.w << 16); z[7] = __uint_as_float(r.w & 0xffff0000u);
     }
     static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    // Largest element of n vectors (NaNs are passed over, as fmaxf does): two elements per instruction on the packed
+    // words, the exact same value as a maximum over the unpacked floats.
+    static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b)
+    {
+        uint32_t d;
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+        return d;
+    }
+    template <int N> static __device__ __forceinline__ float vec_max(const uint4 (&r)[N])
+    {
+        uint32_t m = max2(max2(r[0].x, r[0].y), max2(r[0].z, r[0].w));
+#pragma unroll
+        for (int u = 1; u < N; ++u) m = max2(m, max2(max2(r[u].x, r[u].y), max2(r[u].z, r[u].w)));
+        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+    }
 };
 template <> struct Elems<POLYSPEC_F32> {
     static constexpr int per_vec = 4;
@@ -109,6 +124,14 @@ template <> struct Elems<POLYSPEC_F32> {
         z[2] = __uint_as_float(r.z); z[3] = __uint_as_float(r.w);
     }
     static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    template <int N> static __device__ __forceinline__ float vec_max(const uint4 (&r)[N])
+    {
+        float m = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < N; ++u)
+            m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(r[u].x), __uint_as_float(r[u].y)), fmaxf(__uint_as_float(r[u].z), __uint_as_float(r[u].w))));
+        return m;
+    }
 };
 
 // Where work item `item` lives: first byte and byte count of its row segment.
@@ -230,13 +253,9 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
             }
             float z[kVecPerLane][EPV];
             if (MODE == 0) {
-                float M = -INFINITY;
+                const float M = EL::vec_max(r);
 #pragma unroll
-                for (int u = 0; u < kVecPerLane; ++u) {
-                    EL::unpack(r[u], z[u]);
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) M = fmaxf(M, z[u][e]);
-                }
+                for (int u = 0; u < kVecPerLane; ++u) EL::unpack(r[u], z[u]);
                 const float En = (M == -INFINITY) ? kEmptyRef : ceilf(M * c);
                 if (En > E) {
                     const float sc = pow2_neg(E - En);
