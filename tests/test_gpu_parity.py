@@ -369,3 +369,27 @@ def test_committed_tokens_follow_the_target_distribution(n_models):
     assert n1 > B // 20
     chi2 = ((c1 - n1 * p1) ** 2 / (n1 * p1)).sum()
     assert chi2 < sps.chi2.ppf(1 - 1e-6, V - 1), (n_models, "second", chi2)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("T,scale,shift", [(0.05, 6.0, 0.0), (0.3, 40.0, 900.0), (5.0, 0.5, -3000.0), (1.0, 200.0, 0.0)])
+def test_level_extreme_temperatures_scales_and_offsets(oracle, dtype, T, scale, shift):
+    """Very peaked and very flat rows, and rows carrying a large common offset: the partial normalisers then differ
+    by hundreds of powers of two between segments of one row (rebased exactly or dropped to zero), and a common
+    offset must change nothing at all."""
+    B, k, V = 96, 4, 20480 + 8
+    g = torch.Generator(device=DEV).manual_seed(int(T * 100) + int(scale))
+    lp = (torch.randn((B, k + 1, V), generator=g, device=DEV) * scale + shift).to(dtype)
+    lq = (lp[:, :k].float() + 0.3 * scale * torch.randn((B, k, V), generator=g, device=DEV)).to(dtype)
+    probs = torch.softmax(lq.double() / T, dim=-1).float()
+    tok = torch.multinomial(probs.reshape(B * k, V), 1, generator=g).reshape(B, k).to(torch.int32)
+    u = torch.from_numpy(synth.philox_uniforms(5, 1, B, k + 1)[0]).to(DEV)
+    out = _np(binding.polyspec_verify_level(lp, lq, tok, u, T, want_probs=True))
+    ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), T, threads=8)
+    assert out["device_status"][0] == 0
+    counts, bad = H.compare_level_batch(out["accepted_len"], out["next_token"], ora)
+    _assert_parity(counts, bad, B * (k + 1), f"extreme T={T} scale={scale} shift={shift} {dtype}")
+    m = np.isfinite(ora["p_at"])
+    # |z c| reaches the thousands here: ex2.approx's argument carries 24 bits, so the relative error grows with it
+    tol = (1e-5 if dtype == torch.float32 else 2e-3) + 2.0 ** -22 * (abs(shift) + 6 * scale) / T
+    np.testing.assert_allclose(out["p_at_draft"][m], ora["p_at"][m], rtol=tol, atol=1e-30)
