@@ -393,3 +393,38 @@ def test_level_extreme_temperatures_scales_and_offsets(oracle, dtype, T, scale, 
     # |z c| reaches the thousands here: ex2.approx's argument carries 24 bits, so the relative error grows with it
     tol = (1e-5 if dtype == torch.float32 else 2e-3) + 2.0 ** -22 * (abs(shift) + 6 * scale) / T
     np.testing.assert_allclose(out["p_at_draft"][m], ora["p_at"][m], rtol=tol, atol=1e-30)
+
+
+def test_level_and_chain_random_shapes(oracle):
+    """Forty seeded draws of (batch, block lengths, vocabulary, number of models, type, temperature, per-sequence
+    block lengths): shapes nobody picked by hand, each against the oracle."""
+    rng = np.random.default_rng(20251026)
+    total = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0}
+    for case in range(40):
+        n_models = int(rng.integers(2, 6))
+        B = int(rng.integers(1, 70))
+        V = 8 * int(rng.integers(1, 700))
+        k = tuple(int(x) for x in rng.integers(1, 13, size=n_models - 1))
+        if case % 8 == 0:
+            k = k[:-1] + (32,)                                   # the longest block at the bottom now and then
+        dtype = torch.float32 if rng.random() < 0.5 else torch.bfloat16
+        T = float(rng.choice([0.5, 0.8, 1.0, 1.7]))
+        sig = tuple(float(x) for x in rng.uniform(0.3, 2.5, size=n_models - 1))
+        spec = synth.ChainSpec(f"rand{case}", n_models, B, V, dtype, k, T, 2.5, sig, bool(rng.random() < 0.5))
+        d = synth.make_chain(spec, seed=1000 + case, device=DEV)
+        out = _run_chain(d)
+        ora = _oracle_chain(oracle, d, threads=8)
+        counts, bad = H.compare_chain(out, ora)
+        assert not bad, (case, n_models, B, V, k, dtype, T, bad[:3])
+        for key in total:
+            total[key] += counts[key]
+        if n_models == 2:                                        # the single-level call with ragged block lengths
+            bl = torch.from_numpy(rng.integers(0, k[0] + 1, size=B).astype(np.int32)).to(DEV)
+            lv = _np(binding.polyspec_verify_level(d["models"][0], d["models"][1][:, : k[0]].contiguous(), d["draft_tokens"],
+                                                   d["uniforms"][0].contiguous(), T, block_len=bl))
+            ol = oracle.verify_level(d["models"][0].cpu(), d["models"][1].cpu(), d["draft_tokens"].cpu(), d["uniforms"][0].cpu(), T,
+                                     block_len=bl.cpu())
+            c2, bad2 = H.compare_level_batch(lv["accepted_len"], lv["next_token"], ol)
+            assert not bad2, (case, B, V, k, bad2[:3])
+    print(f"[parity] random shapes: {total}")
+    assert total["tie_accept"] + total["tie_sample"] <= 4
