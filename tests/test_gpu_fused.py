@@ -157,3 +157,35 @@ def test_halves_of_the_fused_call_equal_the_whole_call():
     torch.cuda.synchronize()
     assert torch.equal(again["accepted_len"], whole["accepted_len"]) and torch.equal(again["next_token"], whole["next_token"])
     assert int(call.device_status.item()) == 0
+
+
+def test_lm_head_random_shapes(oracle):
+    """Twenty-four seeded draws of (rows, vocabulary, depth): tile edges nobody picked by hand."""
+    rng = np.random.default_rng(2510)
+    for case in range(24):
+        rows = int(rng.integers(1, 640))
+        V = 4 * int(rng.integers(1, 1500))
+        d = 64 * int(rng.integers(1, 17))
+        h, W = _gemm_case(rows, V, d, seed=9000 + case)
+        out, status = binding.polyspec_lm_head(h, W)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref = oracle.lm_head_logits(h, W)
+        bound = torch.matmul(h.double().abs().cpu(), W.double().abs().cpu().t())
+        worst = float(((out.double().cpu() - ref).abs() / bound.clamp(min=1e-30)).max())
+        assert worst < 16 * 2.0 ** -24, (case, rows, V, d, worst)
+
+
+def test_fused_random_shapes(oracle):
+    """Twelve seeded draws of the fused call's sizes (batch, block, vocabulary, both depths), each against the oracle."""
+    rng = np.random.default_rng(26527)
+    for case in range(12):
+        k = int(rng.integers(1, 13))
+        B = int(rng.integers(1, 1 + 560 // (k + 1)))
+        V = 8 * int(rng.integers(16, 700))
+        d_q = 64 * int(rng.integers(1, 5))
+        d_p = d_q + 64 * int(rng.integers(1, 6))
+        spec = synth.FusedSpec(B=B, k=k, V=V, d_p=d_p, d_q=d_q)
+        d = synth.make_fused(spec, seed=300 + case, device=DEV)
+        print(f"[fused random] case {case}: B={B} k={k} V={V} d_p={d_p} d_q={d_q}")
+        _fused_compare(oracle, d, lambda dl: 4 * dl / spec.temperature)
