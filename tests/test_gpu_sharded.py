@@ -244,3 +244,25 @@ def test_chain_unusable_input_below_reports_minus_one_above():
     for key in CHAIN_KEYS:
         w = want[key].cpu().numpy()
         assert (got[key][:, [2, 4]] == w[:, [2, 4]]).all(), key          # the same report as the unsharded call
+
+
+def test_chain_random_shapes_and_rank_counts(oracle):
+    """Sixteen seeded draws of (models, batch, blocks, slice size, ranks, type), each against the oracle's chain."""
+    rng = np.random.default_rng(4052)
+    for case in range(16):
+        n_models = int(rng.integers(2, 5))
+        R = int(rng.choice([1, 2, 3, 4, 6, 8]))
+        B = int(rng.integers(1, 40))
+        V = R * 8 * int(rng.integers(1, 300))
+        k = tuple(int(x) for x in rng.integers(1, 11, size=n_models - 1))
+        dtype = torch.float32 if rng.random() < 0.5 else torch.bfloat16
+        sig = tuple(float(x) for x in rng.uniform(0.3, 2.0, size=n_models - 1))
+        spec = synth.ChainSpec(f"rs{case}", n_models, B, V, dtype, k, float(rng.choice([0.6, 1.0, 1.5])), 2.5, sig, True)
+        d = synth.make_chain(spec, seed=2000 + case, device=DEV)
+        got, status = _run_sharded_chain(d, R)
+        assert status == 0
+        ora = oracle.verify_chain([m.cpu() for m in d["models"]], d["k"], d["draft_tokens"].cpu(), d["uniforms"].cpu(),
+                                  d["temperature"], threads=8)
+        counts, bad = H.compare_chain(got, ora)
+        assert not bad, (case, n_models, R, B, V, k, dtype, bad[:3])
+        assert counts["tie_accept"] + counts["tie_sample"] <= 1, (case, counts)
