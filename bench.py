@@ -3,23 +3,26 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5|cfg3|cfg2|cfg1|cfg4] [--impl reference]
 
-`--workload cfg4` is the fused path (hidden states -> LM-head projections on the tensor cores -> verification); its
-roofline object is the tensor one.
-
-One step = one pass of the whole hot path (row statistics over every logits row of every model,
-then accept tests / first rejection / replacement-or-bonus sampling / hand-off for every level)
-over one batch that is already resident in HBM.  The default workload is the largest logits-path
+One step = one pass of the whole hot path (the temperature-softmax normaliser of every logits row of
+every model, accept tests, first rejection, replacement-or-bonus sampling and hand-off for every level)
+over one batch that is already resident in HBM.  The headline workload is the largest logits-path
 configuration, the four-level chain (B=256 per GPU, V=152064, bf16, k=(10,6,4) bottom-up, 2.57 GB of
-logits per call -- larger than L2, so nothing is served from cache between steps).
+logits per call -- larger than L2, so nothing is served from cache between steps).  `--workload cfg4` is
+the fused path (hidden states -> LM-head projections on the tensor cores -> verification); its roofline
+object is the tensor one.
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle as it stands on the host
-cores on a bounded sample of the same workload.
+Prints ONE JSON line (rank 0).  A default run (one GPU, headline workload) also measures the four other
+configurations for a fixed number of steps each and embeds their records under "workloads"; every record
+carries the parity counters of its timed batch against the CPU oracle.  `--gpus N` launches N ranks (one
+per GPU, independent replicas) unless a launcher already did.  `--impl reference` times the CPU oracle
+as it stands on the host cores on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -30,16 +33,18 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 from paper_2510_26527_b200 import synth  # noqa: E402
 
 METRIC = "verified_draft_tokens_per_s"
 UNIT = "tokens/s"
+TIE_BAND = 1e-6
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-statistics kernel, from the ncu
-# capture summarised under profiles/ (bytes per logits byte processed, measured on a smaller case of
-# the same kernel and scaled by the bytes one launch processes).  None until a capture exists.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel that streams the logits, from the
+# ncu capture summarised under profiles/ (bytes per logits byte processed, measured on a smaller case of
+# the same kernel and scaled by the bytes one launch processes).  None once the kernel has changed since.
 STATS_TRAFFIC_PER_LOGIT_BYTE = 1.0130     # profiles/stats_kernel_bf16_cfg3_ncu_full.md: (328.350 + 4.250) MB moved for 328.340 MB of logits
 # the same counters per launch of the LM-head kernel on the fused workload
 # (profiles/lmhead_kernel_cfg4_ncu.md: 402.98 MB read + 53.81 MB written)
@@ -134,43 +139,90 @@ def verified_tokens(block_len) -> int:
     return int(block_len.clamp(min=0).sum().item())
 
 
+def spread(ms):
+    """mean / median / min of a list of per-step times in milliseconds."""
+    return {"mean": float(np.mean(ms)), "median": float(np.median(ms)), "min": float(np.min(ms))}
+
+
+# ----------------------------------------------------------------------------------------- parity of the timed batch
+def _classify(ga, gn, oa, on, margin, sinfo):
+    """One (level, sequence) result against the oracle's: exact, a counted tie (a uniform within 1e-6 of its
+    decision threshold, and for a sample the neighbouring positive-mass token), or a mismatch."""
+    if ga == oa and gn == on:
+        return "exact"
+    if ga != oa:
+        j = min(ga, oa)
+        if 0 <= j < len(margin) and np.isfinite(margin[j]) and margin[j] <= TIE_BAND:
+            return "tie_accept"
+        return "mismatch"
+    if sinfo[0] <= TIE_BAND and gn >= 0 and gn in (int(sinfo[2]), int(sinfo[3])):
+        return "tie_sample"
+    return "mismatch"
+
+
+def parity_chain(gpu, ora):
+    """Counters over every (level, sequence) of a chain batch, bottom level first; after a tie the two sides walk
+    different streams, so the levels above it are not compared."""
+    L, B = ora["accepted_len"].shape
+    c = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "skipped_after_tie": 0, "compared": 0}
+    for b in range(B):
+        for l in range(L - 1, -1, -1):
+            ga, oa = int(gpu["accepted_len"][l, b]), int(ora["accepted_len"][l, b])
+            kind = _classify(ga, int(gpu["out_tokens"][l, b, max(ga, 0)]), oa, int(ora["out_tokens"][l, b, max(oa, 0)]),
+                             ora["accept_margin"][l, b], ora["sample_info"][l, b])
+            if kind == "exact" and not (gpu["block_len"][l, b] == ora["block_len"][l, b] and gpu["out_len"][l, b] == ora["out_len"][l, b]
+                                        and (gpu["out_tokens"][l, b] == ora["out_tokens"][l, b]).all()):
+                kind = "mismatch"
+            c[kind] += 1
+            c["compared"] += 1
+            if kind != "exact":
+                if kind != "mismatch":
+                    c["skipped_after_tie"] += l
+                break
+    return c
+
+
+def parity_level(gpu_a, gpu_next, ora):
+    c = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "compared": 0}
+    for b in range(len(ora["accepted_len"])):
+        c[_classify(int(gpu_a[b]), int(gpu_next[b]), int(ora["accepted_len"][b]), int(ora["next_token"][b]),
+                    ora["accept_margin"][b], ora["sample_info"][b])] += 1
+        c["compared"] += 1
+    return c
+
+
 # ----------------------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample(spec, seed, n_seq, device):
-    """The first n_seq sequences of the recipe (same V, rows, dtype), as CPU tensors."""
-    d = synth.make_chain(synth.scaled(spec, B=n_seq), seed=seed, device=device)
-    return {"models": [m.cpu() for m in d["models"]], "k": d["k"], "draft_tokens": d["draft_tokens"].cpu(),
-            "uniforms": d["uniforms"].cpu(), "temperature": d["temperature"]}
-
-
-def oracle_time(sample, threads):
+def oracle_chain(sample, threads):
     from oracle import oracle as orc
     t0 = time.perf_counter()
     out = orc.verify_chain(sample["models"], sample["k"], sample["draft_tokens"], sample["uniforms"],
                            sample["temperature"], threads=threads)
     dt = time.perf_counter() - t0
-    return int(out["block_len"].clip(min=0).sum()), dt
+    return int(out["block_len"].clip(min=0).sum()), dt, out
 
 
-def cpu_baseline(data, spec, target_seconds=12.0):
-    """The oracle, as it stands, on the resident batch: whole passes over it until about target_seconds of CPU work."""
+def cpu_baseline(data, spec, gpu_out, target_seconds=12.0):
+    """The oracle, as it stands, on the resident batch: whole passes over it until about target_seconds of CPU
+    work.  The first pass's outputs are compared with the GPU's outputs on the same batch (parity counters)."""
     from oracle import oracle as orc
     orc.build()
     cores = os.cpu_count() or 1
     sample = {"models": [m.cpu() for m in data["models"]], "k": data["k"], "draft_tokens": data["draft_tokens"].cpu(),
               "uniforms": data["uniforms"].cpu().contiguous(), "temperature": data["temperature"]}
-    tok0, t0 = oracle_time(sample, cores)
+    tok0, t0, out0 = oracle_chain(sample, cores)
+    parity = parity_chain({k: v.cpu().numpy() for k, v in gpu_out.items() if k != "device_status"}, out0)
     passes = int(min(200, max(1, round(target_seconds / max(t0, 1e-3)))))
-    tok, t = 0, 0.0
-    for _ in range(passes):
-        a, b = oracle_time(sample, cores)
+    tok, t = tok0, t0
+    for _ in range(passes - 1):
+        a, b, _ = oracle_chain(sample, cores)
         tok += a
         t += b
     return {"value": tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"{passes} passes over the {spec.B} sequences of the same batch, {tok} verified tokens in {t:.2f} s, "
-                      f"{cores} threads (one sequence per thread)"}
+                      f"{cores} threads (one sequence per thread at a time)"}, parity
 
 
-def fused_oracle_time(d, n_seq, threads):
+def fused_oracle(d, n_seq, threads):
     from oracle import oracle as orc
     t0 = time.perf_counter()
     out = orc.verify_from_hidden(d["hidden_p"][:n_seq], d["W_p"], d["hidden_q"][:n_seq], d["W_q"], d["draft_tokens"][:n_seq].cpu(),
@@ -179,22 +231,39 @@ def fused_oracle_time(d, n_seq, threads):
     return int(n_seq * d["draft_tokens"].shape[1]), dt, out
 
 
-def fused_cpu_baseline(d, spec, target_seconds=12.0):
-    """The oracle's float64 projection + verification on the first sequences of the batch."""
-    from oracle import oracle as orc
-    orc.build()
-    cores = os.cpu_count() or 1
-    n0 = min(spec.B, 2)
-    tok0, t0, _ = fused_oracle_time(d, n0, cores)
-    n = int(min(spec.B, max(n0, n0 * target_seconds / max(t0, 1e-3))))
-    tok, t, _ = fused_oracle_time(d, n, cores)
-    return {"value": tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n} of {spec.B} sequences of the same batch (float64 matmul of the LM head on the host, then the "
-                      f"verification rule), {tok} verified tokens in {t:.2f} s, {cores} threads"}
+def fused_parity(got_a, got_next, logits_p_gpu, ora, d):
+    """Strict counters (1e-6 band) plus, for the disagreements, how many the tensor core's fp32 accumulation
+    explains: an accept uniform within 4 dl / T of min(1, P/Q), or a sampling uniform within 8 dl / (T S) of the GPU
+    token's CDF interval under the oracle's logits (dl = measured max |logit difference|, S = residual mass)."""
+    from scipy.special import softmax as sp_softmax
+    c = parity_level(got_a, got_next, ora)
+    dl = float((logits_p_gpu.double().cpu() - ora["logits_p"]).abs().max())
+    T = d["temperature"]
+    k = d["draft_tokens"].shape[1]
+    u = d["uniforms"].cpu().numpy()
+    band = max(4 * dl / T, TIE_BAND)
+    explained = unexplained = 0
+    for b in range(len(got_a)):
+        ga, gn, oa, on = int(got_a[b]), int(got_next[b]), int(ora["accepted_len"][b]), int(ora["next_token"][b])
+        if ga == oa and gn == on:
+            continue
+        if ga != oa:
+            ok = ora["accept_margin"][b, min(ga, oa)] <= band
+        else:
+            P = sp_softmax(ora["logits_p"][b, oa].numpy() / T)
+            w = np.maximum(P - sp_softmax(ora["logits_q"][b, oa].numpy() / T), 0.0) if oa < k else P
+            cdf = np.cumsum(w)
+            lo, hi = (cdf[gn] - w[gn]) / cdf[-1], cdf[gn] / cdf[-1]
+            ok = w[gn] > 0 and max(lo - u[b, k], u[b, k] - hi, 0.0) <= 2 * band / w.sum()
+        explained += bool(ok)
+        unexplained += not ok
+    c.update({"max_abs_logit_difference": dl, "explained_by_fp32_accumulation": explained, "unexplained": unexplained})
+    return c
 
 
 def run_reference(args, spec):
-    """--impl reference: the CPU oracle on a bounded sample per step."""
+    """--impl reference: the CPU oracle, every step a whole pass over a bounded sample of the workload (several
+    sequences per thread, so that a step does not wait on its slowest sequence alone)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
@@ -206,11 +275,13 @@ def run_reference(args, spec):
         n_seq = min(spec.B, 4)
         d = synth.make_fused(spec, seed=args.seed, device=dev)
         d = {k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}
-        step = lambda: fused_oracle_time(d, n_seq, cores)[:2]
+        step = lambda: fused_oracle(d, n_seq, cores)[:2]
     else:
-        n_seq = min(spec.B, cores)          # one sequence per thread: a step of some tens of milliseconds
-        sample = oracle_sample(spec, seed=args.seed, n_seq=n_seq, device=dev)
-        step = lambda: oracle_time(sample, cores)
+        n_seq = min(spec.B, 4 * cores)
+        d = synth.make_chain(synth.scaled(spec, B=n_seq), seed=args.seed, device=dev)
+        sample = {"models": [m.cpu() for m in d["models"]], "k": d["k"], "draft_tokens": d["draft_tokens"].cpu(),
+                  "uniforms": d["uniforms"].cpu(), "temperature": d["temperature"]}
+        step = lambda: oracle_chain(sample, cores)[:2]
     for _ in range(args.warmup):
         step()
     tokens, elapsed = 0, 0.0
@@ -223,9 +294,9 @@ def run_reference(args, spec):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * elapsed / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(args, spec), "sample": f"{n_seq} sequences per step"},
+        "config": {"workload": workload_name(args, spec)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{n_seq} of {spec.B} sequences of the recipe per step, {args.steps} steps"},
+                         "sample": f"the first {n_seq} of {spec.B} sequences of the recipe per step, {args.steps} steps, {cores} threads"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -257,192 +328,208 @@ def reduce_over_ranks(times_ms, work, device, world):
 
 
 # ----------------------------------------------------------------------------------------- GPU arm
-def run_gpu(args, spec):
-    from paper_2510_26527_b200 import binding, buildlib
-    import torch.distributed as dist
+class Env:
+    """Rank, device and process group of this process (one process per GPU)."""
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: libpolyspec has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0:
-        buildlib.build()
-    if world > 1:
-        dist.barrier()
-    binding.load_library()
-
-    def barrier():
-        if world > 1:
+    def __init__(self):
+        from paper_2510_26527_b200 import binding, buildlib
+        import torch.distributed as dist
+        self.dist = dist
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise RuntimeError("bench.py needs a CUDA device: libpolyspec has no CPU path")
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=self.dev)
+        if self.rank == 0:
+            buildlib.build()
+        if self.world > 1:
             dist.barrier()
+        binding.load_library()
+        self.binding = binding
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
         torch.cuda.synchronize()
 
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def timed_region(env, calls, parts_of, steps, sample_clocks):
+    """K steps between two events, step i on calls[i % len(calls)], with an event after every part of a step
+    (parts_of(call) -> list of (name, function)).  Returns total ms, per-step ms, per-part mean ms, clocks."""
+    names = [n for n, _ in parts_of(calls[0])]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(steps)]
+    fns = [[f for _, f in parts_of(c)] for c in calls]
+    sampler = ClockSampler(env.local)
+    env.barrier()
+    if env.rank == 0 and sample_clocks:
+        sampler.start()
+        time.sleep(0.3)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    env.barrier()
+    start.record()
+    for i in range(steps):
+        f = fns[i % len(fns)]
+        ev[i][0].record()
+        for j, fn in enumerate(f):
+            fn()
+            ev[i][j + 1].record()
+    stop.record()
+    env.barrier()
+    total = start.elapsed_time(stop)
+    clocks = sampler.stop() if (env.rank == 0 and sample_clocks) else None
+    per_step = [e[0].elapsed_time(e[-1]) for e in ev]
+    per_part = {n: sum(e[j].elapsed_time(e[j + 1]) for e in ev) / steps for j, n in enumerate(names)}
+    return total, per_step, per_part, clocks
+
+
+def chain_parts(call):
+    return [("row_stats", call.row_stats), ("walk", call.walk)]
+
+
+def measure_chain(env, args, spec, steps, warmup, headline):
+    """One logits-path workload on this rank's own batch.  Returns the record (rank 0) of the JSON line."""
+    binding, dev, rank, world = env.binding, env.dev, env.rank, env.world
     # sequences are independent: each rank verifies its own batch, no data-path collective
     data = synth.make_chain(spec, seed=args.seed, device=dev, batch_offset=rank * spec.B)
     call = binding.ChainCall(data["models"], data["k"], data["draft_tokens"], data["uniforms"], data["temperature"])
     logits_bytes = spec.logits_bytes()
+    fits_l2 = logits_bytes <= 2 * 126e6
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         call.launch()
     torch.cuda.synchronize()
     tokens_per_step = verified_tokens(call.out["block_len"])
     emitted_per_step = int(call.out["out_len"][0].sum().item())
     assert int(call.device_status.item()) == 0
 
-    # ---- device-timed region: K steps, each = row_stats + walk (exactly polyspec_verify_chain), with an
-    # event between the two halves so the dominant kernel's share is measured live
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local)
-    barrier()
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    start.record()
-    for i in range(args.steps):
-        ev[i][0].record()
-        call.row_stats()
-        ev[i][1].record()
-        call.walk()
-        ev[i][2].record()
-    stop.record()
-    barrier()
-    elapsed_ms = start.elapsed_time(stop)
-    clocks = sampler.stop() if rank == 0 else None
-    stats_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
-    walk_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    # ---- device-timed region: K steps, each exactly polyspec_verify_chain (its two halves, with an event between
+    # them so that the dominant kernel's share is measured live)
+    elapsed_ms, per_step, per_part, clocks = timed_region(env, [call], chain_parts, steps, True)
+    stats_ms, walk_ms = per_part["row_stats"], per_part["walk"]
+    # the same steps as single C-ABI calls, no event inside a step
+    whole_ms, whole_steps, _, _ = timed_region(env, [call], lambda c: [("call", c.launch)], steps, False)
 
-    # ---- end to end: the host-buffer entry point, H2D of every input and D2H of every output inside the region
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    host_models = [m.cpu().pin_memory() for m in data["models"]]
-    host_tok, host_u = data["draft_tokens"].cpu().pin_memory(), data["uniforms"].cpu().pin_memory()
-    rows = [int(m.shape[1]) for m in host_models]
-    ws_bytes = binding.polyspec_verify_chain_host_workspace(data["k"], rows, spec.B, spec.V, call.dt)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    host_out = binding.chain_outputs(spec.n_models - 1, spec.B, spec.kmax, "cpu", pin=True)
-    h2d = sum(m.numel() * m.element_size() for m in host_models) + host_tok.numel() * 4 + host_u.numel() * 4
-    d2h = sum(v.numel() * 4 for v in host_out.values()) + 4
-    binding.polyspec_verify_chain_host(host_models, data["k"], host_tok, host_u, data["temperature"], ws, out=host_out)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(e2e_steps):
+    # ---- inputs that fit in L2: also L2-cold, rotating through >= 256 MB of distinct instances of the workload
+    cold = None
+    if fits_l2 and world == 1:
+        n_inst = int(256e6 // logits_bytes) + 1
+        many = synth.make_chain(synth.scaled(spec, B=spec.B * n_inst), seed=args.seed + 1, device=dev)
+        inst = []
+        for i in range(n_inst):
+            s = slice(i * spec.B, (i + 1) * spec.B)
+            inst.append(binding.ChainCall([m[s] for m in many["models"]], many["k"], many["draft_tokens"][s].contiguous(),
+                                          many["uniforms"][:, s].contiguous(), many["temperature"]))
+        for c in inst:
+            c.launch()
+        torch.cuda.synchronize()
+        cold_ms, cold_steps, _, _ = timed_region(env, inst, lambda c: [("call", c.launch)], max(steps, n_inst), False)
+        cold = {"us_per_call": spread([1e3 * x for x in cold_steps]), "instances": n_inst,
+                "distinct_bytes": n_inst * logits_bytes, "steps": max(steps, n_inst)}
+        del inst, many
+
+    # ---- end to end (headline only): the host-buffer entry point, H2D of every input and D2H of every output inside the region
+    e2e = None
+    if headline:
+        e2e_steps = max(1, min(steps, args.e2e_steps))
+        host_models = [m.cpu().pin_memory() for m in data["models"]]
+        host_tok, host_u = data["draft_tokens"].cpu().pin_memory(), data["uniforms"].cpu().pin_memory()
+        rows = [int(m.shape[1]) for m in host_models]
+        ws_bytes = binding.polyspec_verify_chain_host_workspace(data["k"], rows, spec.B, spec.V, call.dt)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        host_out = binding.chain_outputs(spec.n_models - 1, spec.B, spec.kmax, "cpu", pin=True)
+        h2d = sum(m.numel() * m.element_size() for m in host_models) + host_tok.numel() * 4 + host_u.numel() * 4
+        d2h = sum(v.numel() * 4 for v in host_out.values()) + 4
         binding.polyspec_verify_chain_host(host_models, data["k"], host_tok, host_u, data["temperature"], ws, out=host_out)
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    same = all(bool((host_out[k].to(dev) == call.out[k]).all()) for k in ("accepted_len", "block_len", "out_tokens", "out_len"))
-    del ws, host_models
+        env.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            binding.polyspec_verify_chain_host(host_models, data["k"], host_tok, host_u, data["temperature"], ws, out=host_out)
+        e1.record()
+        env.barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        same = all(bool((host_out[k].to(dev) == call.out[k]).all()) for k in ("accepted_len", "block_len", "out_tokens", "out_len"))
+        del ws, host_models
+    else:
+        e2e_ms, e2e_steps, h2d, d2h, same = 0.0, 1, 0, 0, None
 
     # ---- reduce over ranks: max time, summed work
-    (elapsed_ms, e2e_ms, stats_ms, walk_ms), (tokens_all, emitted_all) = reduce_over_ranks(
-        [elapsed_ms, e2e_ms, stats_ms, walk_ms], [tokens_per_step, emitted_per_step], dev, world)
+    (elapsed_ms, whole_ms, e2e_ms, stats_ms, walk_ms), (tokens_all, emitted_all) = reduce_over_ranks(
+        [elapsed_ms, whole_ms, e2e_ms, stats_ms, walk_ms], [tokens_per_step, emitted_per_step], dev, world)
 
-    base = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:      # the CPU baseline is a one-GPU-run extra
-        base = cpu_baseline(data, spec, target_seconds=args.cpu_seconds)
+    base = parity = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:      # the CPU baseline and the parity check are one-GPU-run extras
+        base, parity = cpu_baseline(data, spec, call.out, target_seconds=args.cpu_seconds if headline else 2.0)
 
-    if rank == 0:
-        peaks = read_peaks()
-        ms_per_step = elapsed_ms / args.steps
-        value = tokens_all * args.steps / (elapsed_ms * 1e-3)
-        achieved = logits_bytes / (stats_ms * 1e-3) / 1e9
+    if rank != 0:
+        return None
+    peaks = read_peaks()
+    ms_per_step = elapsed_ms / steps
+    achieved = logits_bytes / (stats_ms * 1e-3) / 1e9
+    traffic = None if STATS_TRAFFIC_PER_LOGIT_BYTE is None else STATS_TRAFFIC_PER_LOGIT_BYTE * logits_bytes
+    rec = {
+        "metric": METRIC, "value": tokens_all * steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": max(warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name(args, spec), "seed": args.seed,
+                   "l2": ("inputs fit in L2: L2-warm timing (the same instance every step); the L2-cold figure is under l2_cold" if fits_l2 else
+                          f"inputs {logits_bytes / 1e9:.3f} GB per step, larger than the 126 MB L2; no flush needed"),
+                   "parallelism": f"{world} independent replicas, batch sharded, no collective"},
+        "gpu_launches": 2 * steps,
+        "step_ms": spread(per_step),
+        "single_call_step_ms": dict(spread(whole_steps), total_over_steps=whole_ms / steps),
+        "emitted_tokens_per_s": emitted_all * steps / (elapsed_ms * 1e-3),
+        "whole_step_gbs": logits_bytes * world / (ms_per_step * 1e-3) / 1e9,
+        "whole_step_frac_of_hbm_peak": logits_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "kernel_ms": {"row_stats": stats_ms, "walk": walk_ms},
+        "roofline": {"bound": "hbm", "kernel": "stats_kernel (row statistics, every logit once)",
+                     "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "traffic": traffic, "peak_source": f"of {peaks['source']}",
+                     "frac_of_nominal_8TBs": achieved / 8000.0},
+        "clocks": clocks,
+    }
+    if cold is not None:
+        rec["l2_cold"] = cold
+    if headline:
         live_copy = copy_probe_gbs(dev)
-        traffic = None if STATS_TRAFFIC_PER_LOGIT_BYTE is None else STATS_TRAFFIC_PER_LOGIT_BYTE * logits_bytes
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": workload_name(args, spec), "seed": args.seed,
-                       "l2": f"inputs {logits_bytes / 1e9:.3f} GB per step, larger than the 126 MB L2; no flush needed"
-                             if logits_bytes > 2 * 126e6 else "inputs fit in L2: L2-warm timing",
-                       "parallelism": f"{world} independent replicas, batch sharded, no collective"},
-            "gpu_launches": 2 * args.steps,
-            "emitted_tokens_per_s": emitted_all * args.steps / (elapsed_ms * 1e-3),
-            "whole_step_gbs": logits_bytes * world / (ms_per_step * 1e-3) / 1e9,
-            "whole_step_frac_of_hbm_peak": logits_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
-            "kernel_ms": {"row_stats": stats_ms, "walk": walk_ms},
-            "roofline": {"bound": "hbm", "kernel": "stats_kernel (row statistics, every logit once)",
-                         "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                         "traffic": traffic, "peak_source": f"of {peaks['source']}",
-                         "frac_of_nominal_8TBs": achieved / 8000.0,
-                         "this_gpu_copy_gbs": live_copy, "frac_of_this_gpu_copy": achieved / live_copy},
-            "e2e": {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
-                    "matches_device_path": same},
-            "clocks": clocks,
-        }
-        if base is not None:
-            line["cpu_baseline"] = base
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+        rec["roofline"].update({"this_gpu_copy_gbs": live_copy, "frac_of_this_gpu_copy": achieved / live_copy})
+        rec["e2e"] = {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                      "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                      "matches_device_path": same}
+    if base is not None:
+        rec["cpu_baseline"] = base
+        rec["parity"] = parity
+    return rec
 
 
-def run_gpu_fused(args, spec):
+def measure_fused(env, args, spec, steps, warmup, headline):
     """cfg4: hidden states -> LM-head projections on the tensor cores -> verification, one C-ABI call per step."""
-    from paper_2510_26527_b200 import binding, buildlib
-    import torch.distributed as dist
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: libpolyspec has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0:
-        buildlib.build()
-    if world > 1:
-        dist.barrier()
-    binding.load_library()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
+    binding, dev, rank, world = env.binding, env.dev, env.rank, env.world
     d = synth.make_fused(spec, seed=args.seed + 7919 * rank, device=dev)
     call = binding.FusedCall(d["hidden_p"], d["W_p"], d["hidden_q"], d["W_q"], d["draft_tokens"], d["uniforms"], d["temperature"])
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         call.launch()
     torch.cuda.synchronize()
     assert int(call.device_status.item()) == 0
     tokens_per_step = spec.B * spec.k
     emitted_per_step = int((call.out["accepted_len"] + 1).sum().item())
 
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local)
-    barrier()
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    start.record()
-    for i in range(args.steps):
-        ev[i][0].record()
-        call.project()
-        ev[i][1].record()
-        call.verify()
-        ev[i][2].record()
-    stop.record()
-    barrier()
-    elapsed_ms = start.elapsed_time(stop)
-    clocks = sampler.stop() if rank == 0 else None
-    gemm_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / args.steps
-    verify_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / args.steps
+    elapsed_ms, per_step, per_part, clocks = timed_region(
+        env, [call], lambda c: [("lm_head_project_with_row_stats", c.project), ("walk", c.verify)], steps, True)
+    gemm_ms, verify_ms = per_part["lm_head_project_with_row_stats"], per_part["walk"]
+    whole_ms, whole_steps, _, _ = timed_region(env, [call], lambda c: [("call", c.launch)], steps, False)
 
     # end to end: this step's hidden states, draft tokens and uniforms come from pinned host memory, the
     # outputs go back to pinned host memory; the LM-head weights are model parameters and stay resident
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_steps = max(1, min(steps, args.e2e_steps))
     host_in = [t.cpu().pin_memory() for t in (d["hidden_p"], d["hidden_q"], d["draft_tokens"], d["uniforms"])]
     dev_in = [d["hidden_p"], d["hidden_q"], d["draft_tokens"], d["uniforms"]]
     host_out = [torch.empty(spec.B, dtype=torch.int32).pin_memory() for _ in range(2)]
@@ -456,55 +543,92 @@ def run_gpu_fused(args, spec):
         host_out[0].copy_(call.out["accepted_len"], non_blocking=True)
         host_out[1].copy_(call.out["next_token"], non_blocking=True)
     e2e_step()
-    barrier()
+    env.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
     e1.record()
-    barrier()
+    env.barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    (elapsed_ms, e2e_ms, gemm_ms, verify_ms), (tokens_all, emitted_all) = reduce_over_ranks(
-        [elapsed_ms, e2e_ms, gemm_ms, verify_ms], [tokens_per_step, emitted_per_step], dev, world)
+    (elapsed_ms, whole_ms, e2e_ms, gemm_ms, verify_ms), (tokens_all, emitted_all) = reduce_over_ranks(
+        [elapsed_ms, whole_ms, e2e_ms, gemm_ms, verify_ms], [tokens_per_step, emitted_per_step], dev, world)
 
-    base = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:      # the CPU baseline is a one-GPU-run extra
-        base = fused_cpu_baseline({k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}, spec, target_seconds=args.cpu_seconds)
+    base = parity = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import oracle as orc
+        orc.build()
+        cores = os.cpu_count() or 1
+        dc = {k: (v.cpu() if torch.is_tensor(v) else v) for k, v in d.items()}
+        tok, t, ora = fused_oracle(dc, spec.B, cores)        # the whole timed batch: parity and the baseline in one pass
+        lp, _ = binding.polyspec_lm_head(d["hidden_p"], d["W_p"])
+        torch.cuda.synchronize()
+        parity = fused_parity(call.out["accepted_len"].cpu().numpy(), call.out["next_token"].cpu().numpy(), lp, ora, dc)
+        base = {"value": tok / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"all {spec.B} sequences of the same batch, once (float64 matmul of the LM head on the host, then the "
+                          f"verification rule), {tok} verified tokens in {t:.2f} s, {cores} threads"}
 
-    if rank == 0:
-        peaks = read_peaks()
-        ms_per_step = elapsed_ms / args.steps
-        flops = spec.flops()
-        achieved = flops / (gemm_ms * 1e-3) / 1e12
-        line = {
-            "metric": METRIC, "value": tokens_all * args.steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": workload_name(args, spec), "seed": args.seed,
-                       "l2": f"inputs {(spec.weight_bytes() + 2 * spec.B * (spec.k + 1) * (spec.d_p + spec.d_q)) / 1e9:.3f} GB per step, "
-                             "larger than the 126 MB L2; no flush needed",
-                       "parallelism": f"{world} independent replicas, batch sharded, no collective"},
-            "gpu_launches": 2 * args.steps,
-            "emitted_tokens_per_s": emitted_all * args.steps / (elapsed_ms * 1e-3),
-            "whole_step_tflops": flops * world / (ms_per_step * 1e-3) / 1e12,
-            "whole_step_frac_of_tensor_peak": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
-            "kernel_ms": {"lm_head_project_with_row_stats": gemm_ms, "walk": verify_ms},
-            "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (both LM-head projections, tcgen05 cta_group::2)",
-                         "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                         "traffic": LMHEAD_TRAFFIC_BYTES, "peak_source": f"of {peaks['source']} (burst)",
-                         "weight_stream_gbs": spec.weight_bytes() / (gemm_ms * 1e-3) / 1e9,
-                         "weight_stream_frac_of_hbm_peak": spec.weight_bytes() / (gemm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
-            "e2e": {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
-                    "note": "hidden states, tokens and uniforms copied per step; LM-head weights resident"},
-            "clocks": clocks,
-        }
-        if base is not None:
-            line["cpu_baseline"] = base
+    if rank != 0:
+        return None
+    peaks = read_peaks()
+    ms_per_step = elapsed_ms / steps
+    flops = spec.flops()
+    achieved = flops / (gemm_ms * 1e-3) / 1e12
+    call_ms = whole_ms / steps
+    rec = {
+        "metric": METRIC, "value": tokens_all * steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": steps, "warmup": max(warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(args, spec), "seed": args.seed,
+                   "l2": f"inputs {(spec.weight_bytes() + 2 * spec.B * (spec.k + 1) * (spec.d_p + spec.d_q)) / 1e9:.3f} GB per step, "
+                         "larger than the 126 MB L2; no flush needed",
+                   "parallelism": f"{world} independent replicas, batch sharded, no collective"},
+        "gpu_launches": 2 * steps,
+        "step_ms": spread(per_step),
+        "single_call_step_ms": dict(spread(whole_steps), total_over_steps=call_ms),
+        "emitted_tokens_per_s": emitted_all * steps / (elapsed_ms * 1e-3),
+        "whole_step_tflops": flops * world / (ms_per_step * 1e-3) / 1e12,
+        "whole_step_frac_of_tensor_peak": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "whole_step_frac_of_sustained_tensor_peak": flops / (ms_per_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "single_call_frac_of_tensor_peak": flops / (call_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "kernel_ms": {"lm_head_project_with_row_stats": gemm_ms, "walk": verify_ms},
+        "roofline": {"bound": "tensor", "kernel": "lmhead_kernel (both LM-head projections, tcgen05 cta_group::2)",
+                     "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                     "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                     "traffic": LMHEAD_TRAFFIC_BYTES, "peak_source": f"of {peaks['source']} (burst)",
+                     "weight_stream_gbs": spec.weight_bytes() / (gemm_ms * 1e-3) / 1e9,
+                     "weight_stream_frac_of_hbm_peak": spec.weight_bytes() / (gemm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "e2e": {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                "note": "hidden states, tokens and uniforms copied per step; LM-head weights resident"},
+        "clocks": clocks,
+    }
+    if base is not None:
+        rec["cpu_baseline"] = base
+        rec["parity"] = parity
+    return rec
+
+
+def run_gpu(args, spec):
+    env = Env()
+    fused = isinstance(spec, synth.FusedSpec)
+    line = (measure_fused if fused else measure_chain)(env, args, spec, args.steps, args.warmup, True)
+    # a default run (one GPU, the headline workload) also measures the other four configurations, briefly
+    if env.world == 1 and args.workload == "cfg5" and args.batch == 0 and not args.no_workloads:
+        others = {}
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4"):
+            torch.cuda.empty_cache()
+            sp = synth.FusedSpec() if name == "cfg4" else chain_spec(name, args.sigma)
+            rec = (measure_fused if name == "cfg4" else measure_chain)(env, args, sp, args.workload_steps, 5, False)
+            for drop in ("metric", "unit", "n_gpus", "higher_is_better", "scaling", "vs_baseline", "data"):
+                rec.pop(drop, None)
+            rec["us_per_step"] = 1e3 * rec["ms_per_step"]
+            others[name] = rec
+        line["workloads"] = others
+    if env.rank == 0:
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    env.close()
 
 
 def run_gpu_greedy(args, spec):
@@ -562,7 +686,40 @@ def run_gpu_greedy(args, spec):
         "clocks": clocks}))
 
 
-def main():
+# ----------------------------------------------------------------------------------------- launcher
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_ranks(n: int, argv) -> int:
+    """`--gpus N` without a launcher: start N ranks of this script (one process per GPU) on this node and
+    return their exit status.  The ranks are independent replicas; they meet only to combine times and counts."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def launch_check():
+    """What a multi-rank run adds on the host, without any kernel: rendezvous, the MAX / SUM reduction and rank 0's
+    single line.  Runs on `gloo` when there is no GPU (the CPU test of the launcher uses it)."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    use_cuda = torch.cuda.is_available()
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0"))) if use_cuda else torch.device("cpu")
+    if world > 1:
+        dist.init_process_group("nccl" if use_cuda else "gloo")
+    (t_max,), (work,) = reduce_over_ranks([10.0 + rank], [100 * (rank + 1)], dev, world)
+    if rank == 0:
+        print(json.dumps({"launch_check": True, "n_gpus": world, "max_ms": t_max, "summed_work": work}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else list(argv)
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
@@ -578,7 +735,14 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+    ap.add_argument("--no-workloads", action="store_true", help="headline workload only")
+    ap.add_argument("--workload-steps", type=int, default=1000, help="steps of each of the other configurations in a default run")
+    ap.add_argument("--launch-check", action="store_true", help="rendezvous and reduction only (no kernels)")
+    args = ap.parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(launch_ranks(args.gpus, argv))
+    if args.launch_check:
+        return launch_check()
     spec = synth.FusedSpec() if args.workload == "cfg4" else chain_spec(args.workload, args.sigma)
     if args.batch > 0 and args.workload != "cfg4":
         spec = synth.scaled(spec, B=args.batch)
@@ -586,8 +750,6 @@ def main():
         run_reference(args, spec)
     elif args.rule == "greedy" and args.workload != "cfg4":
         run_gpu_greedy(args, spec)
-    elif args.workload == "cfg4":
-        run_gpu_fused(args, spec)
     else:
         run_gpu(args, spec)
 

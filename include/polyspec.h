@@ -5,7 +5,7 @@
  * Vocabulary of the paper (Section 3.1, Problem Formulation): a chain of models
  * M_1 (the target) ... M_n (the smallest drafter); p_i(x | x_<=t) is model i's
  * distribution over the vocabulary at a position; M_n drafts a block of tokens that is
- * "verified in ascending order by M_{n-1}, ..., M_1"; the acceptance length of a
+ * checked bottom-up, by M_{n-1} first and M_1 last; the acceptance length of a
  * verifier (Eq. 1) is the number of consecutive block tokens it accepts.  A *level* is
  * one adjacent pair: verifier M_l checking the token stream handed up by M_{l+1}.
  *
@@ -24,8 +24,9 @@
  *
  * Conventions for every call
  *   - All pointers are DEVICE pointers owned by the caller unless a parameter says
- *     "host".  Logits buffers must be 16-byte aligned and V * sizeof(element) must be a
- *     multiple of 16.  Row-major, innermost dimension = vocabulary.
+ *     "host".  Logits buffers must be 16-byte aligned and V must be a multiple of 8 (the
+ *     kernels read logits eight at a time; other V return POLYSPEC_ERR_UNSUPPORTED).
+ *     Row-major, innermost dimension = vocabulary.
  *   - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL is
  *     the default stream) and return; outputs are valid once the stream has synchronised.
  *   - The library allocates no device memory: the caller passes a workspace of at least

@@ -172,7 +172,7 @@ def verify_level(logits_p, logits_q, draft_tokens, uniforms, temperature, block_
 
 
 def verify_chain(models, k, draft_tokens, uniforms, temperature, bottom_len=None, threads=1, seqs=None):
-    """The chain over a batch (Section 3.1: verified in ascending order by M_{n-1} ... M_1).
+    """The chain over a batch (Section 3.1: checked bottom-up, by M_{n-1} first and M_1 last).
 
     models[i] is [B, rows_i, V] (models[0] = M_1, the target; models[-1] = M_n, the drafter),
     k[l] the largest block level l verifies (l = 0 is M_1's level), draft_tokens

@@ -12,8 +12,8 @@
  * What follows the paper, and where:
  *   - the model chain M_1 (target) ... M_n and the per-position distributions
  *     p_i(x | x_<=t) over the vocabulary: Section 3.1 (Problem Formulation);
- *   - "M_n drafts a block of K tokens, verified in ascending order by
- *     M_{n-1}, ..., M_1": Section 3.1; this is pso_verify_chain_seq's loop;
+ *   - the block of K tokens drafted by M_n is checked bottom-up, by M_{n-1}
+ *     first and M_1 last: Section 3.1; this is pso_verify_chain_seq's loop;
  *   - Verify(x_i, p_i) with a break at the first failure: Algorithm 1, the inner
  *     for-loop; the verification rule is speculative sampling (Sections 2, 3.1,
  *     3.2), i.e. accept with probability min(1, p/q);
@@ -219,8 +219,8 @@ int pso_verify_level_seq(const void* p_rows, const void* q_rows, int dtype, int6
 }
 
 /*
- * The chain for one sequence (Section 3.1: the block drafted by M_n is "verified in
- * ascending order by M_{n-1}, ..., M_1").  Array index l = 0 .. n-2 is the level whose
+ * The chain for one sequence (Section 3.1: the block drafted by M_n is checked
+ * bottom-up, by M_{n-1} first and M_1 last).  Array index l = 0 .. n-2 is the level whose
  * verifier is model l (model 0 = M_1, the target); the bottom level l = n-2 runs first.
  *
  *   model_rows[i]  first logits row of model i for this sequence, model_nrows[i] rows
@@ -289,8 +289,8 @@ int pso_verify_chain_seq(const void* const* model_rows, const int32_t* model_nro
 }
 
 /*
- * Greedy matching, the other verification rule Section 3.1 names ("speculative sampling,
- * greedy matching, or another verification rule") and the one Section 4.5 compares
+ * Greedy matching, the other verification rule Section 3.1 names beside speculative
+ * sampling, and the one Section 4.5 compares
  * acceptance-length variance against: a block token is accepted iff it is the verifier's
  * most likely token at its position, the loop breaks at the first mismatch, and the
  * token emitted after the accepted prefix is the verifier's most likely token there (at

@@ -473,7 +473,7 @@ polyspec_status polyspec_verify_chain_host(
     polyspec_model_logits dev_models[kMaxModels];
     // bottom-up order: the drafter's rows are the first the kernels touch
     for (int i = n_models - 1; i >= 0; --i) {
-        if (cudaMemcpyAsync(ws + h.logits[i], models_host[i].logits, h.logits_bytes[i], cudaMemcpyHostToDevice, s) != cudaSuccess)
+        if (cuda_failed(cudaMemcpyAsync(ws + h.logits[i], models_host[i].logits, h.logits_bytes[i], cudaMemcpyHostToDevice, s)))
             return POLYSPEC_ERR_CUDA;
         dev_models[i].logits = ws + h.logits[i];
         dev_models[i].rows = rows[i];

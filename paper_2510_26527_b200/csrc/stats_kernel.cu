@@ -17,6 +17,8 @@
 // Every wait on an mbarrier is bounded.  If one expires the warp records
 // POLYSPEC_ERR_TIMEOUT, lets the copies it has in flight land (again bounded) and returns;
 // the outputs of that launch are then meaningless.
+#include <mutex>
+
 #include "polyspec_kernels.cuh"
 
 namespace polyspec {
@@ -316,7 +318,8 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
 }
 
 constexpr int kMaxDevices = 64;
-int g_sm_count[kMaxDevices] = {0};     // per device: SM count, filled together with the kernels' shared-memory opt-in
+std::mutex g_setup_mutex;
+int g_sm_count[kMaxDevices] = {0};     // per device: SM count, published under g_setup_mutex once the kernels' shared-memory opt-in is done
 constexpr size_t kStatsSmemBytes = static_cast<size_t>(kWarps) * kStages * (kChunkBytes + sizeof(unsigned long long));
 
 }  // namespace
@@ -346,6 +349,9 @@ cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t s
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int sm_count = 0;
+    {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (g_sm_count[dev] == 0) {
         int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -360,7 +366,9 @@ cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t s
         }
         g_sm_count[dev] = sms > 0 ? sms : 148;
     }
-    const int grid = p.n_items < g_sm_count[dev] ? p.n_items : g_sm_count[dev];   // one CTA per SM
+    sm_count = g_sm_count[dev];
+    }
+    const int grid = p.n_items < sm_count ? p.n_items : sm_count;   // one CTA per SM
     if (dt == POLYSPEC_BF16) {
         if (argmax) stats_kernel<POLYSPEC_BF16, 1><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);
         else stats_kernel<POLYSPEC_BF16, 0><<<grid, kStatsThreads, kStatsSmemBytes, stream>>>(p);

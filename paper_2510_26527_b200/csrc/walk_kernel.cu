@@ -1,5 +1,5 @@
 // Decision and sampling: one CTA walks one sequence up the chain, level by level
-// (Section 3.1: the drafted block is "verified in ascending order by M_{n-1}, ..., M_1").
+// (Section 3.1: the drafted block is checked bottom-up, by M_{n-1} first and M_1 last).
 // Per level (Algorithm 1: Verify with a break at the first failure, then the token that
 // replaces the first rejected one, or the bonus token after a fully accepted block):
 //   1. merge the row-statistics partials of the rows this level needs;
@@ -14,6 +14,8 @@
 // row pass of step 3 is divided by tile ranges, the shares' sums and the chosen token being exchanged
 // through distributed shared memory around two cluster barriers (hardware barriers that every CTA
 // reaches unconditionally; nothing else waits).
+#include <mutex>
+
 #include "polyspec_kernels.cuh"
 #include "walk_device.cuh"
 
@@ -40,6 +42,12 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
     // (row statistics or the LM-head projection) is still finishing; nothing it wrote is touched before
     // this point.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // A CTA may only touch a peer's shared memory once that peer is known to have started: one cluster
+    // barrier up front, reached by every CTA of the cluster unconditionally.
+    if (p.cluster > 1) {
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
     // blockIdx.x = sequence * cluster size + rank in the cluster; only rank 0 writes results
     ClusterCtx cl;
     cl.size = p.cluster;
@@ -180,7 +188,8 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
 }  // namespace
 
 namespace {
-int g_walk_sms[64] = {0};
+std::mutex g_walk_mutex;
+int g_walk_sms[64] = {0};     // per device, filled once under g_walk_mutex
 }
 
 cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p_in, cudaStream_t stream)
@@ -190,18 +199,23 @@ cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p_in, cudaStream_t 
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (g_walk_sms[dev] == 0) {
-        int sms = 0;
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        g_walk_sms[dev] = sms > 0 ? sms : 148;
+    int walk_sms = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_walk_mutex);
+        if (g_walk_sms[dev] == 0) {
+            int sms = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return e;
+            g_walk_sms[dev] = sms > 0 ? sms : 148;
+        }
+        walk_sms = g_walk_sms[dev];
     }
     const int ntiles = (p_in.V + kTile - 1) / kTile;
     // Few sequences: a cluster of up to 8 CTAs walks each one, so that the row passes use more SMs.
     // The largest power of two that still lets every CTA be resident at once (two per SM).
     WalkParams p = p_in;
     p.cluster = 1;
-    while (p.cluster < 8 && static_cast<long long>(p.B) * (2 * p.cluster) <= 2LL * g_walk_sms[dev] && 2 * p.cluster <= ntiles)
+    while (p.cluster < 8 && static_cast<long long>(p.B) * (2 * p.cluster) <= 2LL * walk_sms && 2 * p.cluster <= ntiles)
         p.cluster *= 2;
     const size_t smem = static_cast<size_t>(ntiles) * sizeof(float);
     cudaLaunchConfig_t cfg = {};

@@ -237,6 +237,67 @@ def test_config5_full_size_sampled_sequences(oracle, sigma):
     assert abs(diff2.mean()) < 3 * se2 + 1e-9, (sigma, diff2.mean(), se2)
 
 
+@pytest.mark.parametrize("seed_index", [0, 1])
+@pytest.mark.parametrize("sigma", synth.CFG5_SIGMAS)
+def test_config5_full_batch_every_sequence_against_the_oracle(oracle, sigma, seed_index):
+    """The launch configuration the benchmark times, all 256 sequences of the batch compared with the oracle one
+    by one (every level, every emitted token), for each inter-level noise and two seeds."""
+    import os
+    spec = synth.config("cfg5", sigma=sigma)
+    d = synth.make_chain(spec, seed=7000 + 100 * seed_index + int(sigma * 4), device=DEV)
+    out = _run_chain(d)
+    ora = _oracle_chain(oracle, d, threads=os.cpu_count() or 8)
+    counts, bad = H.compare_chain(out, ora)
+    _assert_parity(counts, bad, spec.B * sum(spec.k), f"cfg5 sigma={sigma} seed {seed_index}, whole batch")
+    assert out["device_status"][0] == 0
+    assert counts["exact"] + counts["tie_accept"] + counts["tie_sample"] + counts["skipped_after_tie"] == spec.B * 3
+
+
+@pytest.mark.parametrize("sigma", synth.CFG5_SIGMAS)
+def test_config5_sixty_four_seeds_acceptance_length_against_the_closed_form(oracle, sigma):
+    """64 seeded instances per inter-level noise (16384 sequences): the bottom level's accepted length has mean
+    sum_j prod_{i<=j} alpha_i and second moment sum_j (2j-1) prod_{i<=j} alpha_i given the logits, alpha_i = sum_v
+    min(P_i, Q_i) (float64 softmax on the device); the sample mean of the difference must vanish within three standard
+    errors.  The first eight sequences of every instance are also compared with the oracle token by token."""
+    spec = synth.config("cfg5", sigma=sigma)
+    k = spec.k
+    seqs = list(range(8))
+    diffs, diffs2, acc = [], [], [[], [], []]
+    total = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "skipped_after_tie": 0}
+    j = torch.arange(1, k[2] + 1, device=DEV, dtype=torch.float64)
+    for s in range(64):
+        d = synth.make_chain(spec, seed=9000 + s, device=DEV)
+        out = _run_chain(d)
+        assert out["device_status"][0] == 0
+        sub = [m[seqs].cpu() for m in d["models"]]
+        ora = oracle.verify_chain(sub, d["k"], d["draft_tokens"][seqs].cpu(), d["uniforms"][:, seqs].cpu().contiguous(),
+                                  spec.temperature, threads=8)
+        counts, bad = H.compare_chain({key: out[key][:, seqs] for key in ("accepted_len", "block_len", "out_tokens", "out_len")}, ora)
+        assert not bad, (sigma, s, bad[:3])
+        for key in total:
+            total[key] += counts[key]
+        P = torch.softmax(d["models"][2][:, :k[2]].double(), dim=-1)
+        Q = torch.softmax(d["models"][3].double(), dim=-1)
+        surv = torch.cumprod(torch.minimum(P, Q).sum(-1), dim=1)
+        del P, Q
+        a = out["accepted_len"][2].astype(np.float64)
+        diffs.append(a - surv.sum(1).cpu().numpy())
+        diffs2.append(a * a - ((2 * j - 1) * surv).sum(1).cpu().numpy())
+        for l in range(3):
+            acc[l].append(out["accepted_len"][l].astype(np.float64))
+        del d
+    diff, diff2 = np.concatenate(diffs), np.concatenate(diffs2)
+    se, se2 = diff.std(ddof=1) / np.sqrt(len(diff)), diff2.std(ddof=1) / np.sqrt(len(diff2))
+    means = [float(np.concatenate(acc[l]).mean()) for l in range(3)]
+    var = [float(np.concatenate(acc[l]).var(ddof=1)) for l in range(3)]
+    print(f"[cfg5-stats] sigma={sigma}: {len(diff)} sequences; mean accepted_len M3/M2/M1 levels = {means[2]:.4f}/{means[1]:.4f}/{means[0]:.4f}, "
+          f"variance {var[2]:.4f}/{var[1]:.4f}/{var[0]:.4f}; bottom level mean - closed form = {diff.mean():+.5f} (se {se:.5f}), "
+          f"second moment - closed form = {diff2.mean():+.5f} (se {se2:.5f}); oracle on 8 sequences per instance: {total}")
+    assert abs(diff.mean()) < 3 * se + 1e-9, (sigma, diff.mean(), se)
+    assert abs(diff2.mean()) < 3 * se2 + 1e-9, (sigma, diff2.mean(), se2)
+    assert total["tie_accept"] + total["tie_sample"] <= max(2, 64 * 8 * 20 // 2000)
+
+
 def test_chain_host_entry_point_matches_device_entry_point():
     spec = synth.scaled(synth.config("cfg5", sigma=1.0), B=16, V=16384)
     d = synth.make_chain(spec, seed=9, device=DEV)

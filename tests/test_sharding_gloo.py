@@ -62,3 +62,33 @@ def test_two_gloo_ranks_shard_and_reduce(tmp_path):
     assert not np.array_equal(u[0], u[1])
     # every rank did real work
     assert r[0][0] > 0 and r[1][0] > 0
+
+
+def _bench(*argv, timeout=300):
+    import subprocess
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    env.pop("WORLD_SIZE", None)
+    env.pop("RANK", None)
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *argv], capture_output=True, text=True,
+                          timeout=timeout, env=env, cwd=ROOT)
+
+
+def test_bench_gpus_flag_launches_that_many_ranks():
+    """`bench.py --gpus 2` starts two ranks itself (no outer launcher): they rendezvous, reduce times with MAX and
+    work with SUM, and rank 0 alone prints the line, with n_gpus = 2.  Run here on `gloo` without any kernel."""
+    import json
+    res = _bench("--gpus", "2", "--launch-check")
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    assert lines[0] == {"launch_check": True, "n_gpus": 2, "max_ms": 11.0, "summed_work": 300.0}
+
+
+def test_bench_gpus_flag_without_a_gpu_fails_in_every_rank():
+    """No CPU path: without a CUDA device both ranks of `--gpus 2` stop with the library's own error."""
+    if torch.cuda.is_available():
+        import pytest
+        pytest.skip("a CUDA device is present")
+    res = _bench("--gpus", "2", "--steps", "1", "--warmup", "1", "--no-workloads")
+    assert res.returncode != 0
+    assert res.stderr.count("bench.py needs a CUDA device") >= 2, res.stderr[-3000:]
