@@ -145,9 +145,18 @@ def spread(ms):
 
 
 # ----------------------------------------------------------------------------------------- parity of the timed batch
-def _classify(ga, gn, oa, on, margin, sinfo):
-    """One (level, sequence) result against the oracle's: exact, a counted tie (a uniform within 1e-6 of its
-    decision threshold, and for a sample the neighbouring positive-mass token), or a mismatch."""
+def _cdf_distance(w, u, token):
+    """Distance, in normalised CDF units, from u to `token`'s inverse-CDF interval under the weights w (inf for a zero-mass token)."""
+    if token < 0 or token >= len(w) or not (w[token] > 0.0):
+        return float("inf")
+    c = np.cumsum(w)
+    return float(max((c[token] - w[token]) / c[-1] - u, u - c[token] / c[-1], 0.0))
+
+
+def _classify(ga, gn, oa, on, margin, sinfo, distance=None):
+    """One (level, sequence) result against the oracle's: exact, a counted tie (a uniform within 1e-6 of its decision
+    threshold; for a sample the other side's token must be the neighbouring positive-mass token or, where tokens are
+    lighter than the band, one whose own interval lies within 1e-6 of the uniform), or a mismatch."""
     if ga == oa and gn == on:
         return "exact"
     if ga != oa:
@@ -155,21 +164,36 @@ def _classify(ga, gn, oa, on, margin, sinfo):
         if 0 <= j < len(margin) and np.isfinite(margin[j]) and margin[j] <= TIE_BAND:
             return "tie_accept"
         return "mismatch"
-    if sinfo[0] <= TIE_BAND and gn >= 0 and gn in (int(sinfo[2]), int(sinfo[3])):
-        return "tie_sample"
+    if sinfo[0] <= TIE_BAND and gn >= 0:
+        if gn in (int(sinfo[2]), int(sinfo[3])) or (distance is not None and distance(gn) <= TIE_BAND):
+            return "tie_sample"
     return "mismatch"
 
 
-def parity_chain(gpu, ora):
+def parity_chain(gpu, ora, sample=None):
     """Counters over every (level, sequence) of a chain batch, bottom level first; after a tie the two sides walk
-    different streams, so the levels above it are not compared."""
+    different streams, so the levels above it are not compared.  `sample` (the oracle's inputs) lets a sampling tie
+    among tokens lighter than the band be recognised from the float64 weights of the row pair."""
+    from oracle import oracle as orc
     L, B = ora["accepted_len"].shape
     c = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "skipped_after_tie": 0, "compared": 0}
+
+    def distance_at(l, b):
+        if sample is None:
+            return None
+
+        def distance(token):
+            a, m, T = int(ora["accepted_len"][l, b]), int(ora["block_len"][l, b]), sample["temperature"]
+            P = orc.softmax_row(sample["models"][l][b, a], T)
+            w = np.maximum(P - orc.softmax_row(sample["models"][l + 1][b, a], T), 0.0) if a < m else P
+            return _cdf_distance(w if w.sum() > 0.0 else P, float(sample["uniforms"][l, b, -1]), int(token))
+        return distance
+
     for b in range(B):
         for l in range(L - 1, -1, -1):
             ga, oa = int(gpu["accepted_len"][l, b]), int(ora["accepted_len"][l, b])
             kind = _classify(ga, int(gpu["out_tokens"][l, b, max(ga, 0)]), oa, int(ora["out_tokens"][l, b, max(oa, 0)]),
-                             ora["accept_margin"][l, b], ora["sample_info"][l, b])
+                             ora["accept_margin"][l, b], ora["sample_info"][l, b], distance_at(l, b))
             if kind == "exact" and not (gpu["block_len"][l, b] == ora["block_len"][l, b] and gpu["out_len"][l, b] == ora["out_len"][l, b]
                                         and (gpu["out_tokens"][l, b] == ora["out_tokens"][l, b]).all()):
                 kind = "mismatch"
@@ -210,7 +234,7 @@ def cpu_baseline(data, spec, gpu_out, target_seconds=12.0):
     sample = {"models": [m.cpu() for m in data["models"]], "k": data["k"], "draft_tokens": data["draft_tokens"].cpu(),
               "uniforms": data["uniforms"].cpu().contiguous(), "temperature": data["temperature"]}
     tok0, t0, out0 = oracle_chain(sample, cores)
-    parity = parity_chain({k: v.cpu().numpy() for k, v in gpu_out.items() if k != "device_status"}, out0)
+    parity = parity_chain({k: v.cpu().numpy() for k, v in gpu_out.items() if k != "device_status"}, out0, sample)
     passes = int(min(200, max(1, round(target_seconds / max(t0, 1e-3)))))
     tok, t = tok0, t0
     for _ in range(passes - 1):

@@ -111,13 +111,15 @@ def expected_accept_len_second(P1, P2, Q3, k1, k2):
 TIE_BAND = 1e-6
 
 
-def compare_level(gpu_a, gpu_next, ora_a, ora_next, accept_margin, sample_info, band=TIE_BAND):
+def compare_level(gpu_a, gpu_next, ora_a, ora_next, accept_margin, sample_info, band=TIE_BAND, distance=None):
     """Classify one (level, sequence) result against the oracle.
 
     Returns "exact", "tie_accept" (accept decisions differ at a position whose uniform lies within
-    `band` of min(1, P/Q)), "tie_sample" (same accepted length, GPU token is the neighbouring
-    positive-mass token and the sampling uniform lies within `band`, in normalised CDF units, of
-    the edge between them) or "mismatch".
+    `band` of min(1, P/Q)), "tie_sample" (same accepted length, the sampling uniform lies within
+    `band`, in normalised CDF units, of an edge of the oracle's token's interval, and the GPU token
+    is the neighbouring positive-mass token -- or, where tokens carry less mass than the band itself
+    so that several edges fall inside it, a token whose own interval lies within `band` of the
+    uniform: `distance(token)` gives that distance under the oracle's float64 weights) or "mismatch".
     """
     if gpu_a == ora_a and gpu_next == ora_next:
         return "exact"
@@ -127,16 +129,40 @@ def compare_level(gpu_a, gpu_next, ora_a, ora_next, accept_margin, sample_info, 
             return "tie_accept"
         return "mismatch"
     margin, _, prev, succ = sample_info
-    if margin <= band and gpu_next in (int(prev), int(succ)) and gpu_next >= 0:
-        return "tie_sample"
+    if margin <= band and gpu_next >= 0:
+        if gpu_next in (int(prev), int(succ)):
+            return "tie_sample"
+        if distance is not None and distance(gpu_next) <= band:
+            return "tie_sample"
     return "mismatch"
 
 
-def compare_chain(gpu, ora, seqs=None, band=TIE_BAND):
+def chain_sample_distance(oracle, models, uniforms, temperature, ora, seq_map=None):
+    """distance(l, b)(token) for compare_chain: how far, in normalised CDF units, the sampling uniform of level l,
+    sequence b lies from `token`'s inverse-CDF interval under the oracle's float64 weights (the residual of the row
+    pair at the oracle's accepted length, or the bonus row).  models: CPU tensors [B, rows, V]; seq_map maps the
+    index b of `ora` to the row of `models` / `uniforms` (identity if None)."""
+    kmax = uniforms.shape[-1] - 1
+
+    def at(l, b):
+        def distance(token):
+            bb = b if seq_map is None else seq_map[b]
+            a, m = int(ora["accepted_len"][l, b]), int(ora["block_len"][l, b])
+            P = oracle.softmax_row(models[l][bb, a], temperature)
+            w = np.maximum(P - oracle.softmax_row(models[l + 1][bb, a], temperature), 0.0) if a < m else P
+            if not (w.sum() > 0.0):
+                w = P
+            return cdf_distance(w, float(uniforms[l, bb, kmax]), int(token))
+        return distance
+    return at
+
+
+def compare_chain(gpu, ora, seqs=None, band=TIE_BAND, distance=None):
     """Compare chain outputs (dicts of numpy arrays [L, B, ...]) sequence by sequence, bottom level first.
 
     After a counted tie the two sides walk different streams, so the levels above it are skipped
-    (counted as "skipped_after_tie").  Returns a dict of counts and a list of mismatch descriptions.
+    (counted as "skipped_after_tie").  `distance(l, b)` returns compare_level's distance function
+    (see chain_sample_distance).  Returns a dict of counts and a list of mismatch descriptions.
     """
     L, B = ora["accepted_len"].shape
     counts = {"exact": 0, "tie_accept": 0, "tie_sample": 0, "mismatch": 0, "skipped_after_tie": 0}
@@ -145,7 +171,8 @@ def compare_chain(gpu, ora, seqs=None, band=TIE_BAND):
         for l in range(L - 1, -1, -1):
             kind = compare_level(int(gpu["accepted_len"][l, b]), int(gpu["out_tokens"][l, b, max(int(gpu["accepted_len"][l, b]), 0)]),
                                  int(ora["accepted_len"][l, b]), int(ora["out_tokens"][l, b, max(int(ora["accepted_len"][l, b]), 0)]),
-                                 ora["accept_margin"][l, b], ora["sample_info"][l, b], band)
+                                 ora["accept_margin"][l, b], ora["sample_info"][l, b], band,
+                                 None if distance is None else distance(l, b))
             if kind == "exact":
                 same = (gpu["block_len"][l, b] == ora["block_len"][l, b] and gpu["out_len"][l, b] == ora["out_len"][l, b]
                         and (gpu["out_tokens"][l, b] == ora["out_tokens"][l, b]).all())

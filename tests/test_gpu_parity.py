@@ -246,8 +246,9 @@ def test_config5_full_batch_every_sequence_against_the_oracle(oracle, sigma, see
     spec = synth.config("cfg5", sigma=sigma)
     d = synth.make_chain(spec, seed=7000 + 100 * seed_index + int(sigma * 4), device=DEV)
     out = _run_chain(d)
-    ora = _oracle_chain(oracle, d, threads=os.cpu_count() or 8)
-    counts, bad = H.compare_chain(out, ora)
+    cpu_models = _cpu(d["models"])
+    ora = oracle.verify_chain(cpu_models, d["k"], d["draft_tokens"].cpu(), d["uniforms"].cpu(), d["temperature"], threads=os.cpu_count() or 8)
+    counts, bad = H.compare_chain(out, ora, distance=H.chain_sample_distance(oracle, cpu_models, d["uniforms"].cpu().numpy(), spec.temperature, ora))
     _assert_parity(counts, bad, spec.B * sum(spec.k), f"cfg5 sigma={sigma} seed {seed_index}, whole batch")
     assert out["device_status"][0] == 0
     assert counts["exact"] + counts["tie_accept"] + counts["tie_sample"] + counts["skipped_after_tie"] == spec.B * 3
@@ -272,7 +273,8 @@ def test_config5_sixty_four_seeds_acceptance_length_against_the_closed_form(orac
         sub = [m[seqs].cpu() for m in d["models"]]
         ora = oracle.verify_chain(sub, d["k"], d["draft_tokens"][seqs].cpu(), d["uniforms"][:, seqs].cpu().contiguous(),
                                   spec.temperature, threads=8)
-        counts, bad = H.compare_chain({key: out[key][:, seqs] for key in ("accepted_len", "block_len", "out_tokens", "out_len")}, ora)
+        counts, bad = H.compare_chain({key: out[key][:, seqs] for key in ("accepted_len", "block_len", "out_tokens", "out_len")}, ora,
+                                      distance=H.chain_sample_distance(oracle, sub, d["uniforms"][:, seqs].cpu().numpy(), spec.temperature, ora))
         assert not bad, (sigma, s, bad[:3])
         for key in total:
             total[key] += counts[key]

@@ -368,3 +368,42 @@ def test_fused_variant_is_the_matmul_followed_by_the_level_rule(oracle):
     np.testing.assert_allclose(out["logits_p"].numpy(), ref, rtol=1e-12, atol=1e-12)
     again = oracle.verify_level(out["logits_p"], out["logits_q"][:, :2], d["draft_tokens"], d["uniforms"], 1.0)
     assert (again["accepted_len"] == out["accepted_len"]).all() and (again["next_token"] == out["next_token"]).all()
+
+
+# ---------------------------------------------------------------- tie accounting of the GPU comparisons (host logic)
+def test_sampling_tie_rule_with_tokens_lighter_than_the_band(oracle):
+    """A sampling uniform within 1e-6 of a CDF edge is a counted tie.  Where the tokens next to that edge carry less
+    mass than the band itself, several edges fall inside the band and the other side may land a few tokens away: still
+    a tie if that token's own interval lies within the band of the uniform; never one if it lies further, or if the
+    uniform is not near an edge of the oracle's token at all."""
+    V, T = 64, 1.0
+    z = np.full((1, 2, V), -60.0)
+    z[0, :, 20] = 0.0                      # nearly all of the mass
+    z[0, :, 40] = -0.5
+    z[0, 0, 2:6] = -21.0                   # four tokens of ~5e-10 each at the start of the CDF, where float32 resolves them
+    lq = np.full((1, 1, V), -60.0)
+    lq[0, 0, 63] = 0.0                     # the drafter puts its mass on token 63: the draft is rejected
+    P = H.prob_tables([z[0]], T)[0]
+    Q = H.prob_tables([lq[0]], T)[0]
+    w = np.maximum(P[0] - Q[0], 0.0)
+    cdf = np.cumsum(w) / w.sum()
+    u = np.float32(cdf[3] * (1 + 1e-3))    # just past the edge between tokens 3 and 4
+    U = np.array([[0.999, u]], np.float32)
+    out = oracle.verify_level(z, lq, np.array([[63]], np.int32), U, T)
+    assert out["accepted_len"][0] == 0
+    tok = int(out["next_token"][0])
+    assert tok == 4 and out["sample_info"][0, 0] < 1e-6
+    dist = lambda t: H.cdf_distance(w, float(u), t)
+    margin, info = out["accept_margin"][0], out["sample_info"][0]
+    assert H.compare_level(0, 3, 0, tok, margin, info) == "tie_sample"                     # the neighbour
+    assert H.compare_level(0, 2, 0, tok, margin, info) == "mismatch"                       # adjacency alone: two tokens away
+    assert H.compare_level(0, 2, 0, tok, margin, info, distance=dist) == "tie_sample"      # ... yet within 1e-6 in CDF units
+    assert H.compare_level(0, 20, 0, tok, margin, info, distance=dist) == "tie_sample"     # the heavy token starts 5e-10 away
+    assert H.compare_level(0, 40, 0, tok, margin, info, distance=dist) == "mismatch"       # far in CDF units
+    assert H.compare_level(0, 1, 0, tok, margin, info, distance=dist) == "mismatch"        # a zero-mass token
+    # a uniform in the middle of a heavy token's interval is no tie, whatever the other side returns
+    U2 = np.array([[0.999, 0.3]], np.float32)
+    out2 = oracle.verify_level(z, lq, np.array([[63]], np.int32), U2, T)
+    assert out2["next_token"][0] == 20
+    d2 = lambda t: H.cdf_distance(w, 0.3, t)
+    assert H.compare_level(0, 5, 0, 20, out2["accept_margin"][0], out2["sample_info"][0], distance=d2) == "mismatch"
