@@ -340,6 +340,60 @@ int polyspec_cost_insertion(double T_new, double T_i, double L_new, double L_i, 
                             double* lhs /* host out */, double* rhs /* host out */);
 
 /*
+ * Staged verification with a threshold (Section 3.3, "Staged Verification"; Algorithm 1, three models)
+ * for a batch of independent sequences.  Algorithm 1's loop: M_3 drafts K tokens, M_2 verifies them, what
+ * M_2 hands on joins `accepted` (count `cnt`); once cnt >= mu, M_1 verifies the accumulated block in one
+ * pass, the verified part is committed, t advances, `accepted` and cnt are reset.  Each M_2 round hands on
+ * its whole emitted stream (accepted prefix plus the replacement or bonus token), which is distributed as
+ * M_2's own samples, so the pass of M_1 verifies it against q = M_2's rows and the committed text keeps
+ * M_1's distribution; a round therefore always adds a token.  Accumulation also stops when one more round
+ * might not fit the largest block a level verifies (cnt + K + 1 > POLYSPEC_MAX_K).
+ *
+ * The two verifications of an iteration are ordinary polyspec_verify_level calls (per-sequence block_len);
+ * these calls keep the loop's bookkeeping on the device, so that the loop needs no host read-back per step:
+ *
+ *   polyspec_staged_init          zeroes the state, remaining = B
+ *   per iteration of Algorithm 1's loop, for all sequences at once:
+ *     polyspec_staged_round_begin   -> pos2 [B] (= t + cnt), tokens2 [B, K] (M_3's drafts there), uniforms2 [B, K+1],
+ *                                      block_len2 [B] (K, or 0 for a sequence that is finished)
+ *       -- caller: logits of M_2 at positions pos2 .. pos2+K and of M_3 at pos2 .. pos2+K-1 (the model forwards),
+ *          then polyspec_verify_level(M_2 rows, M_3 rows, tokens2, uniforms2, block_len2) -> accepted_len2, next_token2 --
+ *     polyspec_staged_accumulate    appends each round's stream; where cnt >= mu (or the block is full): pos1 [B] (= t),
+ *                                      tokens1 [B, kcap] (= accepted), uniforms1 [B, kcap+1], block_len1 [B] (= cnt);
+ *                                      block_len1 = 0 elsewhere
+ *       -- caller: logits of M_1 at pos1 .. pos1+kcap and of M_2 at pos1 .. pos1+kcap-1, then
+ *          polyspec_verify_level(M_1 rows, M_2 rows, tokens1, uniforms1, block_len1) -> accepted_len1, next_token1 --
+ *     polyspec_staged_commit        where block_len1 > 0: commits accepted[0 .. a1) and M_1's token, t += a1 + 1,
+ *                                      cnt = 0; a sequence with n_tokens committed is finished
+ *   *remaining (device) counts the sequences still running; a sequence needs at most mu iterations per pass of M_1,
+ *   so reading it back once every mu iterations is at most one read-back per pass.
+ *
+ *   drafts [B, N] int32: M_3's proposal per position (synthetic stand-in: position-indexed);
+ *   u2 [B, R, K+1]: row r serves a sequence's r-th round; u1 [B, C, POLYSPEC_MAX_K+1]: row c serves its c-th pass of
+ *   M_1, slots 0..m-1 the accept tests, slot POLYSPEC_MAX_K the sampling uniform.
+ *   State arrays (device, caller-owned): t, cnt, rounds, cycles, n_committed, done [B]; accepted [B, POLYSPEC_MAX_K];
+ *   committed [B, cap] (-1 where nothing was committed); presented, per_cycle [B, C] (block length and tokens
+ *   committed of each pass); remaining [1].  kcap >= min(POLYSPEC_MAX_K, mu + K).  done: 0 running, else a
+ *   POLYSPEC_STAGED_* code (EXHAUSTED: out of positions N, of uniform rows R / C; BAD_INPUT: a level call reported -1).
+ */
+#define POLYSPEC_STAGED_FINISHED  1
+#define POLYSPEC_STAGED_EXHAUSTED 2
+#define POLYSPEC_STAGED_BAD_INPUT 3
+typedef struct {
+    int B, K, mu, kcap, N, R, C, cap, n_tokens;
+    int32_t *t, *cnt, *rounds, *cycles, *n_committed, *done;
+    int32_t *accepted, *committed, *presented, *per_cycle, *remaining;
+} polyspec_staged_state;
+polyspec_status polyspec_staged_init(const polyspec_staged_state* s /* host */, void* cuda_stream);
+polyspec_status polyspec_staged_round_begin(const polyspec_staged_state* s /* host */, const int32_t* drafts, const float* u2,
+                                            int32_t* pos2, int32_t* tokens2, float* uniforms2, int32_t* block_len2, void* cuda_stream);
+polyspec_status polyspec_staged_accumulate(const polyspec_staged_state* s /* host */, const int32_t* tokens2, const int32_t* block_len2,
+                                           const int32_t* accepted_len2, const int32_t* next_token2, const float* u1,
+                                           int32_t* pos1, int32_t* tokens1, float* uniforms1, int32_t* block_len1, void* cuda_stream);
+polyspec_status polyspec_staged_commit(const polyspec_staged_state* s /* host */, const int32_t* block_len1, const int32_t* accepted_len1,
+                                       const int32_t* next_token1, void* cuda_stream);
+
+/*
  * polyspec_verify_level_static -- polyspec_verify_level without a workspace argument.
  * (The paper has no counterpart to this call; it exists for integration reasons only.)
  *

@@ -36,6 +36,7 @@ EXPORTS = (
     "polyspec_sharded_level_pick",
     "polyspec_sharded_chain_sizes", "polyspec_sharded_chain_stats", "polyspec_sharded_chain_gather",
     "polyspec_sharded_chain_decide", "polyspec_sharded_chain_pick", "polyspec_sharded_chain_handoff",
+    "polyspec_staged_init", "polyspec_staged_round_begin", "polyspec_staged_accumulate", "polyspec_staged_commit",
 )
 
 
@@ -50,6 +51,16 @@ class PolyspecError(RuntimeError):
 
 class ModelLogits(ctypes.Structure):
     _fields_ = [("logits", ctypes.c_void_p), ("rows", ctypes.c_int)]
+
+
+STAGED_ARRAYS = ("t", "cnt", "rounds", "cycles", "n_committed", "done", "accepted", "committed", "presented", "per_cycle", "remaining")
+STAGED_FINISHED, STAGED_EXHAUSTED, STAGED_BAD_INPUT = 1, 2, 3
+
+
+class StagedState(ctypes.Structure):
+    """polyspec_staged_state: sizes, then the device pointers of the state arrays in STAGED_ARRAYS order."""
+    _fields_ = [(n, ctypes.c_int) for n in ("B", "K", "mu", "kcap", "N", "R", "C", "cap", "n_tokens")] + \
+               [(n, ctypes.c_void_p) for n in STAGED_ARRAYS]
 
 
 _lib = None
@@ -140,6 +151,15 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_sharded_chain_pick.argtypes = [mlp, ci, cip, ci, f32p, ci, ci, ci, ci, ci, cf, vp, i32p, i32p, vp, sz, vp]
     lib.polyspec_sharded_chain_handoff.restype = ci
     lib.polyspec_sharded_chain_handoff.argtypes = [ci, cip, ci, ci, i32p, i32p, i32p, i32p, i32p, i32p, vp]
+    ssp = ctypes.POINTER(StagedState)
+    lib.polyspec_staged_init.restype = ci
+    lib.polyspec_staged_init.argtypes = [ssp, vp]
+    lib.polyspec_staged_round_begin.restype = ci
+    lib.polyspec_staged_round_begin.argtypes = [ssp, i32p, f32p, i32p, i32p, f32p, i32p, vp]
+    lib.polyspec_staged_accumulate.restype = ci
+    lib.polyspec_staged_accumulate.argtypes = [ssp, i32p, i32p, i32p, i32p, f32p, i32p, i32p, f32p, i32p, vp]
+    lib.polyspec_staged_commit.restype = ci
+    lib.polyspec_staged_commit.argtypes = [ssp, i32p, i32p, i32p, vp]
     _lib = lib
     return lib
 

@@ -1,96 +1,132 @@
-"""Staged verification with a threshold (Section 3.3, "Staged Verification"; Algorithm 1) as a host loop
-around ``polyspec_verify_level``, for one sequence and three models on position-indexed logits.
+"""Staged verification with a threshold (Section 3.3, "Staged Verification"; Algorithm 1) for a batch of
+sequences and three models, driven from Python with all state on the device.
 
-Algorithm 1: M_3 drafts K tokens, M_2 verifies them, and what M_2 lets through is accumulated; once at
-least ``mu`` tokens have accumulated, M_1 verifies the accumulated block in one pass, the accepted part
-is committed and t advances.  Here each M_2 round contributes its whole emitted stream (accepted prefix
-plus the replacement or bonus token), which is distributed as M_2's own samples, so that M_1 can verify
-the accumulated block against q = M_2's rows and the committed text keeps M_1's distribution; a round
-therefore always adds at least one token.  Accumulation also stops when another round could overflow the
-largest block a level may verify.
+Algorithm 1: M_3 drafts K tokens, M_2 verifies them, and what M_2 hands on is accumulated; once at least
+``mu`` tokens have accumulated, M_1 verifies the accumulated block in one pass, the verified part is
+committed and t advances.  One iteration of that loop, for every sequence of the batch at once, is
 
-The loop needs fresh logits after every round, which in a real system are model forwards; with synthetic
-logits indexed by position (row i of every model scores position i, whatever the tokens before it) the
-rows are simply slices, so the whole schedule can be run and measured: tokens committed per M_1 call as a
-function of mu.  All verification arithmetic happens in the backend's ``level`` call (the CUDA library
-through ``GpuLevel``); this module only slices, counts and appends.
+    polyspec_staged_round_begin -> [model forwards] -> polyspec_verify_level (M_2 over M_3's drafts)
+    -> polyspec_staged_accumulate -> [model forward] -> polyspec_verify_level (M_1 over the accumulated
+    block, block_len = 0 for the sequences still below the threshold) -> polyspec_staged_commit
+
+and nothing in it comes back to the host: the loop reads one device counter (sequences still running) once
+every ``mu`` iterations, which is at most once per pass of M_1 for any sequence.  All verification and all
+bookkeeping run in the library's kernels; this module only sequences the calls and stands in for the model
+forwards.
+
+The stand-in: logits are indexed by position (row i of every model scores position i, whatever the tokens
+before it), so "running M_2 on positions s .. s+K" is a gather of rows s .. s+K of its table, done here with
+torch indexing on the device positions the library hands out.  That makes the whole schedule runnable and
+measurable on synthetic logits: tokens committed per M_1 pass as a function of mu.
 """
 from __future__ import annotations
 
-from dataclasses import dataclass, field
-from typing import List
+import ctypes
+from typing import Dict
 
 import torch
 
-MAX_BLOCK = 32          # POLYSPEC_MAX_K
+from . import binding
+
+MAX_BLOCK = binding.MAX_K
 
 
-class GpuLevel:
-    """Backend that runs one sequence's level on the GPU through polyspec_verify_level."""
+class StagedBatch:
+    """Device state of Algorithm 1's loop for B sequences, and the loop itself.
 
-    def __init__(self, temperature: float):
-        from . import binding
-        self.binding = binding
-        self.temperature = float(temperature)
-
-    def level(self, rows_p: torch.Tensor, rows_q: torch.Tensor, tokens: torch.Tensor, uniforms: torch.Tensor):
-        """rows_p [m+1, V], rows_q [m, V], tokens [m] int32, uniforms [m+1] float32 (device) -> (accepted, next)."""
-        out = self.binding.polyspec_verify_level(rows_p.unsqueeze(0), rows_q.unsqueeze(0), tokens.unsqueeze(0),
-                                                 uniforms.unsqueeze(0), self.temperature)
-        res = torch.stack([out["accepted_len"][0], out["next_token"][0], out["device_status"][0]]).tolist()   # one sync
-        if res[2] != 0 or res[0] < 0:
-            raise RuntimeError(f"polyspec_verify_level reported device status {res[2]}")
-        return int(res[0]), int(res[1])
-
-
-@dataclass
-class StagedResult:
-    committed: List[int] = field(default_factory=list)      # the text M_1 committed, in order
-    m1_calls: int = 0
-    m2_calls: int = 0
-    per_cycle: List[int] = field(default_factory=list)      # tokens committed by each M_1 call
-    presented: List[int] = field(default_factory=list)      # block length presented to each M_1 call
-
-    @property
-    def tokens_per_m1_call(self) -> float:
-        return len(self.committed) / max(self.m1_calls, 1)
-
-
-def staged_decode(backend, M1: torch.Tensor, M2: torch.Tensor, M3: torch.Tensor, drafts: torch.Tensor,
-                  u2: torch.Tensor, u1: torch.Tensor, K: int, mu: int, n_tokens: int) -> StagedResult:
-    """Run Algorithm 1's schedule from position 0 until ``n_tokens`` are committed.
-
-    M1, M2, M3   [N, V] logits by position (one sequence)
-    drafts       [N] int32: the token M_3 proposes at each position
-    u2           [rounds, K+1] uniforms of the M_2 rounds (row r for the r-th round overall)
-    u1           [cycles, MAX_BLOCK+1] uniforms of the M_1 calls (slots 0..m-1 accept tests, slot MAX_BLOCK sampling)
+    M1, M2, M3   [B, N, V] logits by position (bf16 or fp32, CUDA)
+    drafts       [B, N] int32: the token M_3 proposes at each position
+    u2           [B, R, K+1] float32: row r serves a sequence's r-th M_2 round
+    u1           [B, C, MAX_BLOCK+1] float32: row c serves its c-th M_1 pass (slots 0..m-1 accept tests, slot MAX_BLOCK sampling)
     """
-    if not (1 <= K <= MAX_BLOCK - 1 and 1 <= mu <= MAX_BLOCK):
-        raise ValueError("need 1 <= K < 32 and 1 <= mu <= 32")
-    res = StagedResult()
-    t = 0
-    N = M1.shape[0]
-    while len(res.committed) < n_tokens:
-        acc: List[int] = []
-        # accumulate M_2-verified streams until the threshold (or until another round might not fit)
-        while len(acc) < mu and len(acc) + K + 1 <= MAX_BLOCK:
-            s = t + len(acc)
-            if s + K + 1 > N or res.m2_calls >= u2.shape[0]:
-                raise ValueError("ran out of positions or uniforms")
-            a2, nxt = backend.level(M2[s:s + K + 1], M3[s:s + K], drafts[s:s + K], u2[res.m2_calls])
-            res.m2_calls += 1
-            acc.extend(int(x) for x in drafts[s:s + a2].tolist())
-            acc.append(nxt)
-        m = len(acc)
-        if res.m1_calls >= u1.shape[0]:
-            raise ValueError("ran out of uniforms")
-        u = torch.cat([u1[res.m1_calls, :m], u1[res.m1_calls, MAX_BLOCK:MAX_BLOCK + 1]])
-        block = torch.tensor(acc, dtype=torch.int32, device=M1.device)
-        a1, nxt1 = backend.level(M1[t:t + m + 1], M2[t:t + m], block, u)
-        res.m1_calls += 1
-        res.presented.append(m)
-        res.per_cycle.append(a1 + 1)
-        res.committed.extend(acc[:a1])
-        res.committed.append(nxt1)
-        t += a1 + 1
-    return res
+
+    def __init__(self, M1, M2, M3, drafts, u2, u1, K: int, mu: int, n_tokens: int, temperature: float):
+        self.lib = binding.load_library()
+        for t in (M1, M2, M3, drafts, u2, u1):
+            if not t.is_cuda or not t.is_contiguous():
+                raise ValueError("StagedBatch takes contiguous CUDA tensors")
+        self.M1, self.M2, self.M3, self.drafts, self.u2, self.u1 = M1, M2, M3, drafts, u2, u1
+        B, N, V = M1.shape
+        if tuple(u2.shape[::2]) != (B, K + 1) or tuple(u1.shape[::2]) != (B, MAX_BLOCK + 1) or tuple(drafts.shape) != (B, N):
+            raise ValueError("shapes must be drafts [B,N], u2 [B,R,K+1], u1 [B,C,MAX_BLOCK+1]")
+        self.B, self.N, self.V, self.K, self.mu = B, N, V, int(K), int(mu)
+        self.kcap = min(MAX_BLOCK, self.mu + self.K)
+        self.R, self.C = int(u2.shape[1]), int(u1.shape[1])
+        self.n_tokens = int(n_tokens)
+        self.cap = self.n_tokens + MAX_BLOCK + 1
+        self.temperature = float(temperature)
+        dev = M1.device
+        i32 = lambda *shape: torch.empty(shape, dtype=torch.int32, device=dev)
+        self.state = {name: i32(B) for name in ("t", "cnt", "rounds", "cycles", "n_committed", "done")}
+        self.state.update(accepted=i32(B, MAX_BLOCK), committed=i32(B, self.cap), presented=i32(B, self.C),
+                          per_cycle=i32(B, self.C), remaining=i32(1))
+        self.cstate = binding.StagedState(B, self.K, self.mu, self.kcap, N, self.R, self.C, self.cap, self.n_tokens,
+                                          *[self.state[n].data_ptr() for n in binding.STAGED_ARRAYS])
+        # inputs and outputs of the two level calls of an iteration, allocated once
+        self.pos2, self.block_len2, self.tokens2 = i32(B), i32(B), i32(B, self.K)
+        self.uniforms2 = torch.empty((B, self.K + 1), dtype=torch.float32, device=dev)
+        self.pos1, self.block_len1, self.tokens1 = i32(B), i32(B), i32(B, self.kcap)
+        self.uniforms1 = torch.empty((B, self.kcap + 1), dtype=torch.float32, device=dev)
+        self.out2 = {"accepted_len": i32(B), "next_token": i32(B)}
+        self.out1 = {"accepted_len": i32(B), "next_token": i32(B)}
+        dt = binding._dt(M1)
+        self.ws2 = binding._workspace(binding.polyspec_verify_level_workspace(B, self.K, V, dt), dev)
+        self.ws1 = binding._workspace(binding.polyspec_verify_level_workspace(B, self.kcap, V, dt), dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self._b = torch.arange(B, device=dev).unsqueeze(1)
+        self._ar2 = torch.arange(self.K + 1, device=dev).unsqueeze(0)
+        self._ar1 = torch.arange(self.kcap + 1, device=dev).unsqueeze(0)
+        self.iterations = 0
+        self.read_backs = 0
+        self._check(self.lib.polyspec_staged_init(ctypes.byref(self.cstate), binding._stream(None)), "polyspec_staged_init")
+
+    @staticmethod
+    def _check(st, where):
+        if st != binding.OK:
+            raise binding.PolyspecError(st, where)
+
+    def _forward(self, table, pos, ar):
+        """Stand-in for a model forward: the rows of a position-indexed logits table from `pos` on, per sequence."""
+        idx = (pos.long().unsqueeze(1) + ar).clamp_(max=self.N - 1)
+        return table[self._b, idx]
+
+    def iteration(self):
+        """One pass through the body of Algorithm 1's loop for every sequence; enqueues only."""
+        lib, s, p, q = self.lib, ctypes.byref(self.cstate), binding._ptr, binding._stream(None)
+        self._check(lib.polyspec_staged_round_begin(s, p(self.drafts), p(self.u2), p(self.pos2), p(self.tokens2), p(self.uniforms2),
+                                                    p(self.block_len2), q), "polyspec_staged_round_begin")
+        rows_p = self._forward(self.M2, self.pos2, self._ar2)
+        rows_q = self._forward(self.M3, self.pos2, self._ar2[:, : self.K])
+        binding.polyspec_verify_level(rows_p, rows_q, self.tokens2, self.uniforms2, self.temperature, block_len=self.block_len2,
+                                      workspace=self.ws2, out=self.out2, device_status=self.status)
+        self._check(lib.polyspec_staged_accumulate(s, p(self.tokens2), p(self.block_len2), p(self.out2["accepted_len"]),
+                                                   p(self.out2["next_token"]), p(self.u1), p(self.pos1), p(self.tokens1),
+                                                   p(self.uniforms1), p(self.block_len1), q), "polyspec_staged_accumulate")
+        rows_p = self._forward(self.M1, self.pos1, self._ar1)
+        rows_q = self._forward(self.M2, self.pos1, self._ar1[:, : self.kcap])
+        binding.polyspec_verify_level(rows_p, rows_q, self.tokens1, self.uniforms1, self.temperature, block_len=self.block_len1,
+                                      workspace=self.ws1, out=self.out1, device_status=self.status)
+        self._check(lib.polyspec_staged_commit(s, p(self.block_len1), p(self.out1["accepted_len"]), p(self.out1["next_token"]), q),
+                    "polyspec_staged_commit")
+        self.iterations += 1
+
+    def run(self, max_iterations: int = 100000) -> Dict[str, torch.Tensor]:
+        """Iterate until every sequence has committed n_tokens (or ran out of positions / uniforms)."""
+        while self.iterations < max_iterations:
+            for _ in range(self.mu):
+                self.iteration()
+            self.read_backs += 1
+            if int(self.state["remaining"].item()) == 0:            # the loop's only read-back
+                break
+        return self.results()
+
+    def results(self) -> Dict[str, torch.Tensor]:
+        torch.cuda.synchronize()
+        out = {k: v.cpu() for k, v in self.state.items()}
+        out["iterations"], out["read_backs"] = self.iterations, self.read_backs
+        return out
+
+
+def staged_decode_batch(M1, M2, M3, drafts, u2, u1, K, mu, n_tokens, temperature) -> Dict[str, torch.Tensor]:
+    """Algorithm 1 from position 0 for every sequence of the batch; see StagedBatch."""
+    return StagedBatch(M1, M2, M3, drafts, u2, u1, K, mu, n_tokens, temperature).run()
