@@ -53,6 +53,8 @@ struct ChainArgs {
     size_t workspace_bytes;
     cudaStream_t stream;
     int parts_override;     // > 0: the partials were written by the LM-head projection, this many per row
+    uint32_t spin_limit;    // 0: default; otherwise the try_wait attempts a copy wait may take (test hook)
+    bool single_launch;     // take the single-launch path whatever the row length
 };
 
 polyspec_status check_chain_shape(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt,
@@ -75,8 +77,16 @@ polyspec_status check_chain_shape(int n_models, const int* k, const int* rows, i
     }
     const StatsPlan pl = plan_stats(acc, V, dt);
     if (pl.n_items > 0x7fffffffLL) return POLYSPEC_ERR_UNSUPPORTED;
+    if (plan_chain(acc, B, V, L, dt).q_cap == 0) return POLYSPEC_ERR_UNSUPPORTED;
     *total_rows = acc;
     return POLYSPEC_OK;
+}
+
+// Bytes a chain call needs: the partials (all the two halves use) followed by the single-launch path's counters,
+// per-sequence state, job queue and tile sums.
+size_t chain_workspace_bytes(long long total_rows, int n_models, int B, int V, polyspec_dtype dt)
+{
+    return plan_chain(total_rows, B, V, n_models - 1, dt).total;
 }
 
 // Checks shared by both halves; fills the plan and the row table.
@@ -103,6 +113,7 @@ polyspec_status prepare_chain(const ChainArgs& a, StatsPlan* pl, StatsParams* sp
     sp->c = static_cast<float>(kLog2e / static_cast<double>(a.temperature));
     sp->partials = static_cast<float2*>(a.workspace);
     sp->status = a.device_status;
+    sp->spin_limit = a.spin_limit;
     return POLYSPEC_OK;
 }
 
@@ -117,18 +128,12 @@ polyspec_status run_stats(const ChainArgs& a)
     return POLYSPEC_OK;
 }
 
-// Second half: accept tests, first rejection, replacement / bonus token, hand-off, level by level.
-polyspec_status run_walk(const ChainArgs& a)
+void fill_walk_params(const ChainArgs& a, const StatsParams& sp, int parts, WalkParams* out)
 {
-    StatsPlan pl;
-    StatsParams sp;
-    polyspec_status st = prepare_chain(a, &pl, &sp);
-    if (st != POLYSPEC_OK) return st;
-    if (!a.draft_tokens || !a.uniforms || !a.accepted_len) return POLYSPEC_ERR_INVALID_ARG;
-    WalkParams wp;
+    WalkParams& wp = *out;
     wp.t = sp.t;
     wp.V = a.V;
-    wp.parts = pl.parts;
+    wp.parts = parts;
     wp.c = sp.c;
     wp.partials = sp.partials;
     wp.n_levels = a.n_models - 1;
@@ -150,16 +155,54 @@ polyspec_status run_walk(const ChainArgs& a)
     wp.p_at = a.p_at;
     wp.q_at = a.q_at;
     wp.device_status = a.device_status;
+    wp.cluster = 1;
+}
+
+// Second half: accept tests, first rejection, replacement / bonus token, hand-off, level by level.
+polyspec_status run_walk(const ChainArgs& a)
+{
+    StatsPlan pl;
+    StatsParams sp;
+    polyspec_status st = prepare_chain(a, &pl, &sp);
+    if (st != POLYSPEC_OK) return st;
+    if (!a.draft_tokens || !a.uniforms || !a.accepted_len) return POLYSPEC_ERR_INVALID_ARG;
+    WalkParams wp;
+    fill_walk_params(a, sp, pl.parts, &wp);
     if (cuda_failed(launch_walk(a.dt, wp, a.stream))) return POLYSPEC_ERR_CUDA;
     return POLYSPEC_OK;
 }
 
-polyspec_status run_chain(const ChainArgs& a)
+// The two halves one after the other on the caller's stream (two launches).
+polyspec_status run_chain_two_launch(const ChainArgs& a)
 {
     if (!a.draft_tokens || !a.uniforms || !a.accepted_len) return POLYSPEC_ERR_INVALID_ARG;
     polyspec_status st = run_stats(a);
     if (st != POLYSPEC_OK) return st;
     return run_walk(a);
+}
+
+// Rows shorter than this go through the two launches: what the single launch gains is the second read of a row pair
+// served from L2, which only matters for long rows, while its per-row bookkeeping does not shrink with the row.
+constexpr size_t kSingleLaunchMinRowBytes = 8192;
+
+// The whole chain in one launch: the statistics stream with every sequence's decisions trailing it.
+polyspec_status run_chain(const ChainArgs& a)
+{
+    if (!a.draft_tokens || !a.uniforms || !a.accepted_len) return POLYSPEC_ERR_INVALID_ARG;
+    if (!a.single_launch && static_cast<size_t>(a.V > 0 ? a.V : 0) * elem_size(a.dt) < kSingleLaunchMinRowBytes)
+        return run_chain_two_launch(a);
+    StatsPlan pl;
+    StatsParams sp;
+    polyspec_status st = prepare_chain(a, &pl, &sp);
+    if (st != POLYSPEC_OK) return st;
+    const ChainPlan cp = plan_chain(pl.total_rows, a.B, a.V, a.n_models - 1, a.dt);
+    if (a.workspace_bytes < cp.total) return POLYSPEC_ERR_WORKSPACE;
+    ChainParams p;
+    std::memset(&p, 0, sizeof p);
+    fill_walk_params(a, sp, pl.parts, &p.w);
+    p.spin_limit = a.spin_limit;
+    if (cuda_failed(launch_chain(a.dt, p, cp, a.workspace, a.stream))) return POLYSPEC_ERR_CUDA;
+    return POLYSPEC_OK;
 }
 
 ChainArgs chain_args(const polyspec_model_logits* models, int n_models, const int* k, int B, int V, polyspec_dtype dt,
@@ -202,7 +245,7 @@ const char* polyspec_status_string(polyspec_status s)
     return "unknown status";
 }
 
-int polyspec_version(void) { return 200; }      // 0.2.0: greedy matching, cost model, sharded level added to the ABI
+int polyspec_version(void) { return 300; }      // 0.3.0: single-launch chain, staged verification added to the ABI
 
 const char* polyspec_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
@@ -214,17 +257,17 @@ polyspec_status polyspec_verify_level_workspace(int B, int k, int V, polyspec_dt
     long long total = 0;
     polyspec_status st = check_chain_shape(2, kk, rows, B, V, dt, &total);
     if (st != POLYSPEC_OK) return st;
-    *bytes = plan_stats(total, V, dt).partial_bytes;
+    *bytes = chain_workspace_bytes(total, 2, B, V, dt);
     return POLYSPEC_OK;
 }
 
-polyspec_status polyspec_verify_level(
+namespace {
+ChainArgs level_args(
     const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
     const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
     int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
-    if (!next_token) return POLYSPEC_ERR_INVALID_ARG;
     ChainArgs a;
     std::memset(&a, 0, sizeof a);
     a.logits[0] = logits_p; a.logits[1] = logits_q;
@@ -238,8 +281,61 @@ polyspec_status polyspec_verify_level(
     a.device_status = device_status;
     a.workspace = workspace; a.workspace_bytes = workspace_bytes;
     a.stream = static_cast<cudaStream_t>(cuda_stream);
+    return a;
+}
+}  // namespace
+
+polyspec_status polyspec_verify_level(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
+    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!next_token) return POLYSPEC_ERR_INVALID_ARG;
+    return run_chain(level_args(logits_p, logits_q, draft_tokens, uniforms, block_len, B, k, V, dt, temperature, accepted_len,
+                                next_token, p_at_draft, q_at_draft, device_status, workspace, workspace_bytes, cuda_stream));
+}
+
+polyspec_status polyspec_verify_level_single_launch(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
+    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!next_token) return POLYSPEC_ERR_INVALID_ARG;
+    ChainArgs a = level_args(logits_p, logits_q, draft_tokens, uniforms, block_len, B, k, V, dt, temperature, accepted_len,
+                             next_token, p_at_draft, q_at_draft, device_status, workspace, workspace_bytes, cuda_stream);
+    a.single_launch = true;
     return run_chain(a);
 }
+
+}  // extern "C"
+
+// The level call as two launches (row statistics, then the walk) on a workspace that holds the partials only: what
+// polyspec_verify_level_static runs on its built-in scratch.
+polyspec_status polyspec::verify_level_two_launch_workspace(int B, int k, int V, polyspec_dtype dt, size_t* bytes)
+{
+    const int kk[1] = {k};
+    const int rows[2] = {k + 1, k};
+    long long total = 0;
+    polyspec_status st = check_chain_shape(2, kk, rows, B, V, dt, &total);
+    if (st != POLYSPEC_OK) return st;
+    *bytes = plan_stats(total, V, dt).partial_bytes;
+    return POLYSPEC_OK;
+}
+
+polyspec_status polyspec::verify_level_two_launch(
+    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
+    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!next_token) return POLYSPEC_ERR_INVALID_ARG;
+    return run_chain_two_launch(level_args(logits_p, logits_q, draft_tokens, uniforms, block_len, B, k, V, dt, temperature, accepted_len,
+                                           next_token, p_at_draft, q_at_draft, device_status, workspace, workspace_bytes, cuda_stream));
+}
+
+extern "C" {
 
 polyspec_status polyspec_verify_chain_workspace(int n_models, const int* k, const int* rows, int B, int V,
                                                 polyspec_dtype dt, size_t* bytes)
@@ -248,7 +344,7 @@ polyspec_status polyspec_verify_chain_workspace(int n_models, const int* k, cons
     long long total = 0;
     polyspec_status st = check_chain_shape(n_models, k, rows, B, V, dt, &total);
     if (st != POLYSPEC_OK) return st;
-    *bytes = plan_stats(total, V, dt).partial_bytes;
+    *bytes = chain_workspace_bytes(total, n_models, B, V, dt);
     return POLYSPEC_OK;
 }
 
@@ -265,6 +361,33 @@ polyspec_status polyspec_verify_chain(
     a.accepted_len = accepted_len; a.block_len = block_len; a.out_tokens = out_tokens; a.out_len = out_len;
     a.device_status = device_status;
     return run_chain(a);
+}
+
+polyspec_status polyspec_verify_chain_single_launch(
+    const polyspec_model_logits* models, int n_models, const int* k,
+    const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,
+    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
+    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!models || !k || n_models < 2 || n_models > kMaxModels) return POLYSPEC_ERR_INVALID_ARG;
+    if (!block_len || !out_tokens || !out_len) return POLYSPEC_ERR_INVALID_ARG;
+    ChainArgs a = chain_args(models, n_models, k, B, V, dt, temperature, workspace, workspace_bytes, cuda_stream);
+    a.draft_tokens = draft_tokens; a.uniforms = uniforms;
+    a.accepted_len = accepted_len; a.block_len = block_len; a.out_tokens = out_tokens; a.out_len = out_len;
+    a.device_status = device_status;
+    a.single_launch = true;
+    return run_chain(a);
+}
+
+polyspec_status polyspec_chain_row_stats_wait_limit(
+    const polyspec_model_logits* models, int n_models, const int* k, int B, int V, polyspec_dtype dt,
+    float temperature, unsigned int wait_limit, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!models || !k || n_models < 2 || n_models > kMaxModels || wait_limit == 0) return POLYSPEC_ERR_INVALID_ARG;
+    ChainArgs a = chain_args(models, n_models, k, B, V, dt, temperature, workspace, workspace_bytes, cuda_stream);
+    a.device_status = device_status;
+    a.spin_limit = wait_limit;
+    return run_stats(a);
 }
 
 polyspec_status polyspec_chain_row_stats(
@@ -376,6 +499,7 @@ polyspec_status polyspec_verify_chain_greedy(
     sp.c = 1.0f;
     sp.partials = static_cast<float2*>(workspace);
     sp.status = device_status;
+    sp.spin_limit = 0;
     if (cuda_failed(launch_stats(dt, sp, s, /*argmax=*/true))) return POLYSPEC_ERR_CUDA;
 
     WalkParams wp;
@@ -418,7 +542,7 @@ polyspec_status host_layout(int n_models, const int* k, const int* rows, int B, 
     int kmax = 0;
     for (int l = 0; l < L; ++l) kmax = k[l] > kmax ? k[l] : kmax;
     size_t off = 0;
-    h->partials = off; off += align256(plan_stats(total, V, dt).partial_bytes);
+    h->partials = off; off += align256(chain_workspace_bytes(total, n_models, B, V, dt));
     for (int i = 0; i < n_models; ++i) {
         h->logits_bytes[i] = static_cast<size_t>(B) * rows[i] * V * elem_size(dt);
         h->logits[i] = off; off += align256(h->logits_bytes[i]);

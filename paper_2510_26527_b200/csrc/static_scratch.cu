@@ -50,7 +50,7 @@ polyspec_status polyspec_verify_level_static(
     int32_t* device_status, void* cuda_stream)
 {
     size_t need = 0;
-    const polyspec_status st = polyspec_verify_level_workspace(B, k, V, dt, &need);
+    const polyspec_status st = polyspec::verify_level_two_launch_workspace(B, k, V, dt, &need);
     if (st != POLYSPEC_OK) return st;
     if (need > POLYSPEC_STATIC_SCRATCH_BYTES) return POLYSPEC_ERR_SCRATCH_LIMIT;
     void* scratch = nullptr;
@@ -58,9 +58,9 @@ polyspec_status polyspec_verify_level_static(
     if (ss != POLYSPEC_OK) return ss;
     // Every partial the second kernel reads is written by the first kernel of the same call, so
     // nothing in the array has to start at zero and the previous call's contents are harmless.
-    return polyspec_verify_level(logits_p, logits_q, draft_tokens, uniforms, block_len, B, k, V, dt, temperature,
-                                 accepted_len, next_token, p_at_draft, q_at_draft, device_status,
-                                 scratch, POLYSPEC_STATIC_SCRATCH_BYTES, cuda_stream);
+    return polyspec::verify_level_two_launch(logits_p, logits_q, draft_tokens, uniforms, block_len, B, k, V, dt, temperature,
+                                             accepted_len, next_token, p_at_draft, q_at_draft, device_status,
+                                             scratch, POLYSPEC_STATIC_SCRATCH_BYTES, cuda_stream);
 }
 
 }  // extern "C"

@@ -1,0 +1,124 @@
+// Device helpers of the kernels that stream logits rows through per-warp shared-memory rings with 1-D bulk
+// TMA copies (the row-statistics kernel and the single-launch chain kernel): mbarrier and bulk-copy wrappers
+// with bounded waits, the unpacking of 16-byte vectors, exact power-of-two rescaling.
+#pragma once
+
+#include "polyspec_kernels.cuh"
+
+namespace polyspec {
+namespace streamdev {
+
+constexpr int kChunkBytes = 2048;                 // one bulk copy = one warp-wide sweep of 4 vectors per lane
+#ifndef POLYSPEC_STATS_STAGES
+#define POLYSPEC_STATS_STAGES 2
+#endif
+#ifndef POLYSPEC_STATS_WARPS
+#define POLYSPEC_STATS_WARPS 32
+#endif
+// Measured on the four-level workload: 32 warps x 2 stages 402 us, 28 x 3 410 us, 24 x 4 419 us; warp counts
+// that are not multiples of four (one per scheduler) lose 5 %.
+constexpr int kStages = POLYSPEC_STATS_STAGES;    // per-warp ring depth
+constexpr int kWarps = POLYSPEC_STATS_WARPS;
+constexpr int kStatsThreads = kWarps * 32;
+constexpr int kVecPerLane = kChunkBytes / 16 / 32;   // 4
+constexpr uint32_t kSpinLimit = 1u << 20;         // try_wait attempts before giving up
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kSpinLimit)
+{
+    for (uint32_t i = 0; i < limit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
+{
+    uint4 r;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    return r;
+}
+
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// 2^d for an integer-valued d <= 0 (exact); 0 once below the normal range.
+__device__ __forceinline__ float pow2_neg(float d)
+{
+    return (d < -126.0f) ? 0.0f : __int_as_float((static_cast<int>(d) + 127) << 23);
+}
+
+template <int DT> struct Elems;
+template <> struct Elems<POLYSPEC_BF16> {
+    static constexpr int per_vec = 8;
+    static __device__ __forceinline__ void unpack(const uint4& r, float* z)
+    {
+        z[0] = __uint_as_float(r.x << 16); z[1] = __uint_as_float(r.x & 0xffff0000u);
+        z[2] = __uint_as_float(r.y << 16); z[3] = __uint_as_float(r.y & 0xffff0000u);
+        z[4] = __uint_as_float(r.z << 16); z[5] = __uint_as_float(r.z & 0xffff0000u);
+        z[6] = __uint_as_float(r.w << 16); z[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    // Largest element of n vectors (NaNs are passed over, as fmaxf does): two elements per instruction on the packed
+    // words, the exact same value as a maximum over the unpacked floats.
+    static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b)
+    {
+        uint32_t d;
+        asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+        return d;
+    }
+    template <int N> static __device__ __forceinline__ float vec_max(const uint4 (&r)[N])
+    {
+        uint32_t m = max2(max2(r[0].x, r[0].y), max2(r[0].z, r[0].w));
+#pragma unroll
+        for (int u = 1; u < N; ++u) m = max2(m, max2(max2(r[u].x, r[u].y), max2(r[u].z, r[u].w)));
+        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+    }
+};
+template <> struct Elems<POLYSPEC_F32> {
+    static constexpr int per_vec = 4;
+    static __device__ __forceinline__ void unpack(const uint4& r, float* z)
+    {
+        z[0] = __uint_as_float(r.x); z[1] = __uint_as_float(r.y);
+        z[2] = __uint_as_float(r.z); z[3] = __uint_as_float(r.w);
+    }
+    static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    template <int N> static __device__ __forceinline__ float vec_max(const uint4 (&r)[N])
+    {
+        float m = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < N; ++u)
+            m = fmaxf(m, fmaxf(fmaxf(__uint_as_float(r[u].x), __uint_as_float(r[u].y)), fmaxf(__uint_as_float(r[u].z), __uint_as_float(r[u].w))));
+        return m;
+    }
+};
+
+}  // namespace streamdev
+}  // namespace polyspec

@@ -103,6 +103,9 @@ __device__ __forceinline__ double scale_pow2(double Z, float d)
 // each, keeping a running (E, Z) that is rebased whenever a larger reference turns up; then the
 // lanes are rebased to the warp's largest reference and added.  Rebasing is an exact power-of-two
 // scaling, the sums are in double.  Every lane returns the same result.
+// COHERENT: the partials were written by other SMs during this very launch, so they are read from L2
+// (ld.global.cg) instead of through this SM's L1.
+template <bool COHERENT = false>
 __device__ __forceinline__ RowStat merge_partials(const float2* part, int parts, int lane)
 {
     float E = kEmptyRef;
@@ -112,7 +115,7 @@ __device__ __forceinline__ RowStat merge_partials(const float2* part, int parts,
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int i = i0 + u * 32;
-            ps[u] = (i < parts) ? part[i] : make_float2(kEmptyRef, 0.0f);
+            ps[u] = (i < parts) ? (COHERENT ? __ldcg(part + i) : part[i]) : make_float2(kEmptyRef, 0.0f);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -257,11 +260,12 @@ __device__ __forceinline__ void tiles_pass(const void* prow, const void* qrow, i
 // The token at `target` of the row's running sum, for the warp of the share that contains it: lane i of the warp
 // owns tiles [t0, t1) of the share with sum `mine` and inclusive running sum `incl` over the lanes, `base` is the mass
 // before the share.  Returns the token in every lane (-1 if the share holds no mass).
-template <int DT>
+template <int DT, bool COHERENT = false>
 __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow, int V, float c, float Ep, float iZp, float Eq, float iZq,
                                              bool use_q, const float* tile_sum, int t0, int t1, double mine, double incl,
                                              double base, double target, int lane)
 {
+    auto sum_of = [&](int t) { return COHERENT ? __ldcg(tile_sum + t) : tile_sum[t]; };
     int token = -1;
     const unsigned hit = __ballot_sync(0xffffffffu, base + incl > target);
     const unsigned has_mass = __ballot_sync(0xffffffffu, mine > 0.0);
@@ -274,15 +278,15 @@ __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow,
         if (lane == owner) {
             double run = base + (incl - mine);
             for (int t = t0; t < t1; ++t) {
-                const double nxt = run + static_cast<double>(tile_sum[t]);
+                const double nxt = run + static_cast<double>(sum_of(t));
                 if (nxt > target) { tile = t; prefix = run; break; }
                 run = nxt;
             }
             if (tile < 0) {                       // take the lane's last non-empty tile
                 run = base + (incl - mine);
                 for (int t = t0; t < t1; ++t) {
-                    if (tile_sum[t] > 0.0f) { tile = t; prefix = run; }
-                    run += static_cast<double>(tile_sum[t]);
+                    if (sum_of(t) > 0.0f) { tile = t; prefix = run; }
+                    run += static_cast<double>(sum_of(t));
                 }
             }
         }

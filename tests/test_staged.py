@@ -114,8 +114,9 @@ def test_batched_staged_schedule_on_the_gpu_matches_the_oracle(mu):
     got = run.run()
     assert int(got["remaining"]) == 0 and int(run.status.item()) == 0
     rate = _compare_with_oracle(got, inputs, K, mu, n_tokens, T)
-    # no host read-back per level call: one per mu iterations, i.e. at most one per pass of M_1 of any sequence
-    assert got["read_backs"] * mu == got["iterations"] and got["read_backs"] <= int(got["cycles"].min()) + 1
+    # no host read-back per level call: one per mu iterations, and a pass of M_1 comes after at most mu iterations, so the
+    # loop reads back no more often than the sequence that needed the most passes made them
+    assert got["read_backs"] * mu == got["iterations"] and got["read_backs"] <= int(got["cycles"].max())
     print(f"[staged] mu={mu}: {rate:.2f} tokens per M_1 pass, {float((got['rounds'] / got['cycles']).mean()):.2f} M_2 rounds per pass, "
           f"{got['iterations']} iterations, {got['read_backs']} host read-backs for {B} sequences x {n_tokens} tokens")
 
