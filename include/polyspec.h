@@ -151,27 +151,8 @@ polyspec_status polyspec_chain_walk(
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * How polyspec_verify_level and polyspec_verify_chain run.  Rows of at least 8 KiB take ONE launch: every logits
- * row is streamed once, position by position, and each sequence's decisions (Algorithm 1's accept loop, replacement /
- * bonus token, hand-off) follow as soon as the rows of a position are complete, so that the second read of a row
- * pair -- the residual needs both normalisers first -- is served from L2.  Shorter rows take the two launches of the
- * halves above.  Both give bit-identical results.  The *_single_launch entry points take the single launch whatever
- * the row length (same arguments, same workspace); they exist so that the path can be chosen explicitly.
- */
-polyspec_status polyspec_verify_level_single_launch(
-    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
-    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
-    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
-    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
-polyspec_status polyspec_verify_chain_single_launch(
-    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */,
-    const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,
-    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
-    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
-
-/*
- * polyspec_chain_row_stats_wait_limit -- polyspec_chain_row_stats with the number of polls a warp may spend
- * waiting for one of its copies to land set by the caller (the library's own limit is 2^20 polls).  A diagnostic
+ * polyspec_chain_row_stats_wait_limit -- polyspec_chain_row_stats with the number of looks a warp may take at
+ * the barrier of one of its copies set by the caller (the library's own wait is 2^20 suspending polls).  A diagnostic
  * for the give-up path described in the conventions above: with a limit too small for a copy to land, warps record
  * POLYSPEC_ERR_TIMEOUT in *device_status, still wait (with the full limit) for the copies they have in flight, and
  * return; the workspace contents are then undefined and the device stays usable.  wait_limit >= 1.

@@ -36,7 +36,7 @@ EXPORTS = (
     "polyspec_sharded_level_pick",
     "polyspec_sharded_chain_sizes", "polyspec_sharded_chain_stats", "polyspec_sharded_chain_gather",
     "polyspec_sharded_chain_decide", "polyspec_sharded_chain_pick", "polyspec_sharded_chain_handoff",
-    "polyspec_verify_level_single_launch", "polyspec_verify_chain_single_launch", "polyspec_chain_row_stats_wait_limit",
+    "polyspec_chain_row_stats_wait_limit",
     "polyspec_staged_init", "polyspec_staged_round_begin", "polyspec_staged_accumulate", "polyspec_staged_commit",
 )
 
@@ -104,10 +104,6 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_chain_row_stats.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, i32p, vp, sz, vp]
     lib.polyspec_chain_walk.restype = ci
     lib.polyspec_chain_walk.argtypes = lib.polyspec_verify_chain.argtypes
-    lib.polyspec_verify_chain_single_launch.restype = ci
-    lib.polyspec_verify_chain_single_launch.argtypes = lib.polyspec_verify_chain.argtypes
-    lib.polyspec_verify_level_single_launch.restype = ci
-    lib.polyspec_verify_level_single_launch.argtypes = lib.polyspec_verify_level.argtypes
     lib.polyspec_chain_row_stats_wait_limit.restype = ci
     lib.polyspec_chain_row_stats_wait_limit.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, ctypes.c_uint, i32p, vp, sz, vp]
     lib.polyspec_verify_chain_host_workspace.restype = ci
@@ -220,7 +216,7 @@ def polyspec_verify_level_workspace(B: int, k: int, V: int, dt: int) -> int:
 
 
 def polyspec_verify_level(logits_p, logits_q, draft_tokens, uniforms, temperature, block_len=None,
-                          want_probs=False, workspace=None, out=None, device_status=None, stream=None, single_launch=False):
+                          want_probs=False, workspace=None, out=None, device_status=None, stream=None):
     """One adjacent pair over a batch.  logits_p [B,k+1,V], logits_q [B,k,V], draft_tokens [B,k] int32,
     uniforms [B,k+1] float32; returns device tensors accepted_len [B], next_token [B] (and p_at_draft,
     q_at_draft [B,k] if want_probs) plus the device status word."""
@@ -244,8 +240,7 @@ def polyspec_verify_level(logits_p, logits_q, draft_tokens, uniforms, temperatur
             out["q_at_draft"] = torch.empty((B, k), dtype=torch.float32, device=dev)
     if device_status is None:
         device_status = torch.zeros(1, dtype=torch.int32, device=dev)
-    fn = lib.polyspec_verify_level_single_launch if single_launch else lib.polyspec_verify_level
-    st = fn(
+    st = lib.polyspec_verify_level(
         _ptr(logits_p), _ptr(logits_q), _ptr(draft_tokens), _ptr(uniforms), _ptr(block_len),
         B, k, V, dt, float(temperature), _ptr(out["accepted_len"]), _ptr(out["next_token"]),
         _ptr(out.get("p_at_draft")), _ptr(out.get("q_at_draft")), _ptr(device_status),
@@ -276,7 +271,7 @@ def chain_outputs(L: int, B: int, kmax: int, device, pin=False) -> dict:
 
 
 def polyspec_verify_chain(models, k, draft_tokens, uniforms, temperature, workspace=None, out=None,
-                          device_status=None, stream=None, single_launch=False):
+                          device_status=None, stream=None):
     """n models (models[0] = M_1 ... models[-1] = M_n, each [B, rows_i, V]), n-1 levels verified bottom-up.
     k[l] = largest block level l verifies; draft_tokens [B, k[-1]]; uniforms [n-1, B, max(k)+1]."""
     lib = load_library()
@@ -301,8 +296,7 @@ def polyspec_verify_chain(models, k, draft_tokens, uniforms, temperature, worksp
     if device_status is None:
         device_status = torch.zeros(1, dtype=torch.int32, device=dev)
     arr = (ModelLogits * n)(*[ModelLogits(m.data_ptr(), r) for m, r in zip(models, rows)])
-    fn = lib.polyspec_verify_chain_single_launch if single_launch else lib.polyspec_verify_chain
-    st = fn(arr, n, _int_array(k), _ptr(draft_tokens), _ptr(uniforms), B, V, dt, float(temperature),
+    st = lib.polyspec_verify_chain(arr, n, _int_array(k), _ptr(draft_tokens), _ptr(uniforms), B, V, dt, float(temperature),
                                    _ptr(out["accepted_len"]), _ptr(out["block_len"]), _ptr(out["out_tokens"]),
                                    _ptr(out["out_len"]), _ptr(device_status), _ptr(workspace), workspace.numel(),
                                    _stream(stream))
@@ -399,17 +393,6 @@ class ChainCall:
                                                             int(wait_limit), _ptr(self.device_status), _ptr(self.workspace),
                                                             self.workspace.numel(), _stream(self.stream)),
                "polyspec_chain_row_stats_wait_limit")
-
-    def launch_single(self):
-        _check(self.lib.polyspec_verify_chain_single_launch(self._arr, self.n, self._k, _ptr(self.draft_tokens), _ptr(self.uniforms),
-                                                            self.B, self.V, self.dt, self.temperature, *self._tail()),
-               "polyspec_verify_chain_single_launch")
-        return self.out
-
-    def walk(self):
-        _check(self.lib.polyspec_chain_walk(self._arr, self.n, self._k, _ptr(self.draft_tokens), _ptr(self.uniforms),
-                                            self.B, self.V, self.dt, self.temperature, *self._tail()), "polyspec_chain_walk")
-        return self.out
 
 
 def polyspec_verify_chain_host_workspace(k: Sequence[int], rows: Sequence[int], B: int, V: int, dt: int) -> int:

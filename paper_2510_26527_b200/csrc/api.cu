@@ -54,7 +54,6 @@ struct ChainArgs {
     cudaStream_t stream;
     int parts_override;     // > 0: the partials were written by the LM-head projection, this many per row
     uint32_t spin_limit;    // 0: default; otherwise the try_wait attempts a copy wait may take (test hook)
-    bool single_launch;     // take the single-launch path whatever the row length
 };
 
 polyspec_status check_chain_shape(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt,
@@ -77,16 +76,14 @@ polyspec_status check_chain_shape(int n_models, const int* k, const int* rows, i
     }
     const StatsPlan pl = plan_stats(acc, V, dt);
     if (pl.n_items > 0x7fffffffLL) return POLYSPEC_ERR_UNSUPPORTED;
-    if (plan_chain(acc, B, V, L, dt).q_cap == 0) return POLYSPEC_ERR_UNSUPPORTED;
     *total_rows = acc;
     return POLYSPEC_OK;
 }
 
-// Bytes a chain call needs: the partials (all the two halves use) followed by the single-launch path's counters,
-// per-sequence state, job queue and tile sums.
-size_t chain_workspace_bytes(long long total_rows, int n_models, int B, int V, polyspec_dtype dt)
+// Bytes a chain call needs: the partials.
+size_t chain_workspace_bytes(long long total_rows, int /*n_models*/, int /*B*/, int V, polyspec_dtype dt)
 {
-    return plan_chain(total_rows, B, V, n_models - 1, dt).total;
+    return plan_stats(total_rows, V, dt).partial_bytes;
 }
 
 // Checks shared by both halves; fills the plan and the row table.
@@ -181,28 +178,9 @@ polyspec_status run_chain_two_launch(const ChainArgs& a)
     return run_walk(a);
 }
 
-// Rows shorter than this go through the two launches: what the single launch gains is the second read of a row pair
-// served from L2, which only matters for long rows, while its per-row bookkeeping does not shrink with the row.
-constexpr size_t kSingleLaunchMinRowBytes = 8192;
-
-// The whole chain in one launch: the statistics stream with every sequence's decisions trailing it.
 polyspec_status run_chain(const ChainArgs& a)
 {
-    if (!a.draft_tokens || !a.uniforms || !a.accepted_len) return POLYSPEC_ERR_INVALID_ARG;
-    if (!a.single_launch && static_cast<size_t>(a.V > 0 ? a.V : 0) * elem_size(a.dt) < kSingleLaunchMinRowBytes)
-        return run_chain_two_launch(a);
-    StatsPlan pl;
-    StatsParams sp;
-    polyspec_status st = prepare_chain(a, &pl, &sp);
-    if (st != POLYSPEC_OK) return st;
-    const ChainPlan cp = plan_chain(pl.total_rows, a.B, a.V, a.n_models - 1, a.dt);
-    if (a.workspace_bytes < cp.total) return POLYSPEC_ERR_WORKSPACE;
-    ChainParams p;
-    std::memset(&p, 0, sizeof p);
-    fill_walk_params(a, sp, pl.parts, &p.w);
-    p.spin_limit = a.spin_limit;
-    if (cuda_failed(launch_chain(a.dt, p, cp, a.workspace, a.stream))) return POLYSPEC_ERR_CUDA;
-    return POLYSPEC_OK;
+    return run_chain_two_launch(a);
 }
 
 ChainArgs chain_args(const polyspec_model_logits* models, int n_models, const int* k, int B, int V, polyspec_dtype dt,
@@ -296,19 +274,6 @@ polyspec_status polyspec_verify_level(
                                 next_token, p_at_draft, q_at_draft, device_status, workspace, workspace_bytes, cuda_stream));
 }
 
-polyspec_status polyspec_verify_level_single_launch(
-    const void* logits_p, const void* logits_q, const int32_t* draft_tokens, const float* uniforms,
-    const int32_t* block_len, int B, int k, int V, polyspec_dtype dt, float temperature,
-    int32_t* accepted_len, int32_t* next_token, float* p_at_draft, float* q_at_draft,
-    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
-{
-    if (!next_token) return POLYSPEC_ERR_INVALID_ARG;
-    ChainArgs a = level_args(logits_p, logits_q, draft_tokens, uniforms, block_len, B, k, V, dt, temperature, accepted_len,
-                             next_token, p_at_draft, q_at_draft, device_status, workspace, workspace_bytes, cuda_stream);
-    a.single_launch = true;
-    return run_chain(a);
-}
-
 }  // extern "C"
 
 // The level call as two launches (row statistics, then the walk) on a workspace that holds the partials only: what
@@ -360,22 +325,6 @@ polyspec_status polyspec_verify_chain(
     a.draft_tokens = draft_tokens; a.uniforms = uniforms;
     a.accepted_len = accepted_len; a.block_len = block_len; a.out_tokens = out_tokens; a.out_len = out_len;
     a.device_status = device_status;
-    return run_chain(a);
-}
-
-polyspec_status polyspec_verify_chain_single_launch(
-    const polyspec_model_logits* models, int n_models, const int* k,
-    const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,
-    int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
-    int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
-{
-    if (!models || !k || n_models < 2 || n_models > kMaxModels) return POLYSPEC_ERR_INVALID_ARG;
-    if (!block_len || !out_tokens || !out_len) return POLYSPEC_ERR_INVALID_ARG;
-    ChainArgs a = chain_args(models, n_models, k, B, V, dt, temperature, workspace, workspace_bytes, cuda_stream);
-    a.draft_tokens = draft_tokens; a.uniforms = uniforms;
-    a.accepted_len = accepted_len; a.block_len = block_len; a.out_tokens = out_tokens; a.out_len = out_len;
-    a.device_status = device_status;
-    a.single_launch = true;
     return run_chain(a);
 }
 

@@ -46,7 +46,7 @@ struct StatsParams {
     float c;
     float2* partials;   // [total rows, parts]
     int32_t* status;    // [1] or nullptr: receives POLYSPEC_ERR_TIMEOUT if a bounded wait expires
-    uint32_t spin_limit;   // try_wait attempts of a copy wait before the warp gives up (0: the default, 2^20)
+    uint32_t spin_limit;   // 0: the default wait (2^20 suspending try_waits); otherwise that many non-suspending looks
 };
 
 // Decision + sampling pass: one CTA walks one sequence up the chain.
@@ -91,44 +91,6 @@ cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t s
 cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p, cudaStream_t stream);
 // Greedy matching: reads arg-max partials (launch_stats with argmax = true) of the verifiers' rows only.
 cudaError_t launch_greedy_walk(const WalkParams& p, cudaStream_t stream);
-
-// ---- The whole chain in one launch (chain_kernel.cu): the row-statistics stream and, trailing it by a few
-// microseconds, every sequence's decisions, so that the second read of a row pair comes from L2.
-struct ChainSeqState;      // per-sequence state machine, defined with the kernel
-struct ChainCtl {          // zeroed before every launch
-    int next_item;         // next row segment nobody has claimed yet
-    unsigned int q_head;   // residual jobs: next to hand out
-    unsigned int q_tail;   // residual jobs: reserved so far
-    int finished;          // sequences whose every level is done
-    int pad[12];
-};
-struct ChainParams {
-    WalkParams w;                      // rows, sizes, inputs and outputs, exactly as for the two-launch path
-    int seg;                           // elements per row segment (as StatsParams)
-    int n_items;                       // total rows * parts
-    int pos_begin[kMaxK + 3];          // row slots before position j (position-major order), [max_rows] = total rows
-    int max_rows;                      // largest rows[i]
-    int ntiles, rseg_tiles, n_rsegs;   // sampling tiles per row, tiles per residual job, residual jobs per row pair
-    float2* partials;                  // [total rows, parts] (aliases w.partials, writable)
-    int* row_done;                     // [total rows] segments finished per row
-    ChainSeqState* seq;                // [B]
-    float* tile_sum;                   // [B, ntiles] residual tile sums of the one sample a sequence has in flight
-    unsigned long long* queue;         // [q_cap] residual jobs: (ticket + 1) << 32 | (b * n_rsegs + segment)
-    unsigned int q_cap;
-    ChainCtl* ctl;
-    uint32_t spin_limit;               // try_wait attempts of a copy wait before the warp gives up
-};
-// Workspace of the single-launch path after the partials: everything from `zero_begin` to `zero_end` must be zero at launch.
-struct ChainPlan {
-    StatsPlan stats;
-    size_t row_done, seq, queue, ctl, tile_sum, total;     // byte offsets into the workspace
-    size_t zero_begin, zero_end;
-    unsigned int q_cap;
-    int ntiles, rseg_tiles, n_rsegs;
-};
-ChainPlan plan_chain(long long total_rows, int B, int V, int n_levels, polyspec_dtype dt);
-// Fills the order tables and workspace pointers of `p` (p.w must be complete) and launches; zeroes the control region first.
-cudaError_t launch_chain(polyspec_dtype dt, ChainParams& p, const ChainPlan& plan, void* workspace, cudaStream_t stream);
 
 // The level call as two launches on a workspace that holds the partials only (api.cu); polyspec_verify_level_static
 // runs it on the library's built-in scratch.

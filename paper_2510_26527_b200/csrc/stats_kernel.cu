@@ -127,7 +127,8 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
             __syncwarp();          // every lane has finished reading the stage the next copy will overwrite
             issue_one();
             const uint32_t stage = done % kStages;
-            const bool ok = wait_bounded(smem_u32(&bars[stage]), (done / kStages) & 1u, p.spin_limit ? p.spin_limit : kSpinLimit);
+            const bool ok = p.spin_limit ? wait_polls(smem_u32(&bars[stage]), (done / kStages) & 1u, p.spin_limit)
+                                         : wait_bounded(smem_u32(&bars[stage]), (done / kStages) & 1u);
             if (!__all_sync(0xffffffffu, ok)) {
                 if (lane == 0) {
                     if (p.status) atomicCAS(p.status, 0, static_cast<int>(POLYSPEC_ERR_TIMEOUT));

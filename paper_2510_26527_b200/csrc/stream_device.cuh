@@ -48,6 +48,24 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// One look at the barrier without suspending the thread (try_wait may park it for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// At most `limit` non-suspending looks: the caller-chosen limit of the diagnostic entry point.
+__device__ __forceinline__ bool wait_polls(uint32_t bar, uint32_t parity, uint32_t limit)
+{
+    for (uint32_t i = 0; i < limit; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+    return false;
+}
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kSpinLimit)
 {
     for (uint32_t i = 0; i < limit; ++i)

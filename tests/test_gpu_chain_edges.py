@@ -1,0 +1,80 @@
+"""Edge cases of the chain call on the GPU that the parity file does not reach: unusable input that only an upper
+level meets, a residual that vanishes in floating point, and the give-up path of the row-statistics kernel."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_26527_b200 import binding, buildlib, synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+KEYS = ("accepted_len", "block_len", "out_tokens", "out_len")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    buildlib.build()
+    binding.load_library()
+    assert torch.cuda.is_available()
+
+
+def _np(out):
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def _oracle(oracle, d):
+    return oracle.verify_chain([m.cpu() for m in d["models"]], d["k"], d["draft_tokens"].cpu(), d["uniforms"].cpu(), d["temperature"], threads=8)
+
+
+def test_unusable_row_met_by_an_upper_level_only(oracle):
+    """A NaN in M_2's first row: the bottom level (M_3 over M_4) never sees it and reports normally, M_2's level and
+    M_1's above it report -1, exactly as the oracle does."""
+    spec = synth.scaled(synth.config("cfg5", sigma=0.25), B=6, V=9000)
+    d = synth.make_chain(spec, seed=8, device=DEV)
+    d["models"][1][2, 0, 100] = float("nan")                     # M_2's first row of sequence 2
+    out = _np(binding.polyspec_verify_chain(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"]))
+    ora = _oracle(oracle, d)
+    assert out["device_status"][0] == binding.ERR_BAD_INPUT_ON_DEVICE
+    for key in KEYS:
+        assert (out[key][:, 2] == ora[key][:, 2]).all(), key
+    assert out["accepted_len"][2, 2] >= 0 and out["accepted_len"][1, 2] == -1 and out["accepted_len"][0, 2] == -1
+    counts, bad = H.compare_chain(out, ora, seqs=[0, 1, 3, 4, 5])
+    assert not bad
+
+
+def test_residual_that_vanishes_falls_back_to_the_verifier_row(oracle):
+    """p == q at the rejected row, the rejection forced by an accept uniform above 1: the residual is 0 everywhere and P
+    is sampled instead (the oracle flags the same fall-back)."""
+    g = torch.Generator(device=DEV).manual_seed(3)
+    for Vv in (16384 + 512, 2048):
+        lp = torch.randn((6, 3, Vv), generator=g, device=DEV) * 2
+        lq = lp[:, :2].clone()
+        tok = torch.randint(0, Vv, (6, 2), generator=g, device=DEV, dtype=torch.int32)
+        u = torch.from_numpy(synth.philox_uniforms(4, 1, 6, 3)[0]).to(DEV)
+        u[:, 0] = 1.5
+        out = _np(binding.polyspec_verify_level(lp, lq, tok, u, 1.0))
+        ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), 1.0)
+        assert (ora["fallback"] == 1).all() and (out["accepted_len"] == 0).all()
+        assert (out["next_token"] == ora["next_token"]).all(), (Vv, out["next_token"], ora["next_token"])
+
+
+def test_copy_wait_that_runs_out_reports_timeout_and_leaves_the_device_usable(oracle):
+    """The give-up path of the row-statistics kernel, in the safe form: the wait for a copy is given a single look, which a
+    copy from HBM cannot meet; the warps record POLYSPEC_ERR_TIMEOUT, still wait (full limit) for the copies they
+    have in flight, and return.  The next ordinary call on the same device and workspace is exact."""
+    spec = synth.scaled(synth.config("cfg3"), B=8, V=65536)
+    d = synth.make_chain(spec, seed=17, device=DEV)
+    call = binding.ChainCall(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    call.row_stats_wait_limit(1)
+    torch.cuda.synchronize()
+    assert int(call.device_status.item()) == binding.ERR_TIMEOUT
+    call.device_status.zero_()
+    call.row_stats()
+    out = _np(call.walk())
+    assert out["device_status"][0] == 0
+    counts, bad = H.compare_chain(out, _oracle(oracle, d))
+    assert not bad and counts["exact"] == 8 * 2
+    with pytest.raises(binding.PolyspecError):
+        call.row_stats_wait_limit(0)

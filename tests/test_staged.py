@@ -109,7 +109,7 @@ def test_batched_staged_schedule_on_the_gpu_matches_the_oracle(mu):
     buildlib.build()
     binding.load_library()
     B, V, N, K, T, n_tokens = 24, 4096, 260, 5, 0.9, 120
-    inputs = _gpu_case(B, V, N, K, T, seed=46 + mu, dtype=torch.bfloat16, R=200, C=150)
+    inputs = _gpu_case(B, V, N, K, T, seed=46 + mu, dtype=torch.bfloat16, R=700, C=150)
     run = staged.StagedBatch(*inputs, K, mu, n_tokens, T)
     got = run.run()
     assert int(got["remaining"]) == 0 and int(run.status.item()) == 0
