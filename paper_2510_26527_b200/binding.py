@@ -394,6 +394,11 @@ class ChainCall:
                                                             self.workspace.numel(), _stream(self.stream)),
                "polyspec_chain_row_stats_wait_limit")
 
+    def walk(self):
+        _check(self.lib.polyspec_chain_walk(self._arr, self.n, self._k, _ptr(self.draft_tokens), _ptr(self.uniforms),
+                                            self.B, self.V, self.dt, self.temperature, *self._tail()), "polyspec_chain_walk")
+        return self.out
+
 
 def polyspec_verify_chain_host_workspace(k: Sequence[int], rows: Sequence[int], B: int, V: int, dt: int) -> int:
     n = ctypes.c_size_t(0)
