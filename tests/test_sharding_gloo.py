@@ -92,3 +92,38 @@ def test_bench_gpus_flag_without_a_gpu_fails_in_every_rank():
     res = _bench("--gpus", "2", "--steps", "1", "--warmup", "1", "--no-workloads")
     assert res.returncode != 0
     assert res.stderr.count("bench.py needs a CUDA device") >= 2, res.stderr[-3000:]
+
+
+def test_bench_parity_counters_on_the_host():
+    """bench.py compares the batch it timed with the oracle and reports counters; the comparison itself is host logic:
+    identical outputs are all exact, a changed token away from any CDF edge is a mismatch, a changed accepted length
+    whose uniform sits on the threshold is a counted tie, and levels above a tie are not compared."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from oracle import oracle as orc
+    from paper_2510_26527_b200 import synth
+    spec = synth.scaled(synth.config("cfg5", sigma=0.5), B=5, V=96)
+    d = synth.make_chain(spec, seed=11, device="cpu")
+    ora = orc.verify_chain(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
+    sample = {"models": d["models"], "uniforms": d["uniforms"], "temperature": d["temperature"]}
+    same = {k: ora[k].copy() for k in ("accepted_len", "block_len", "out_tokens", "out_len")}
+    c = bench.parity_chain(same, ora, sample)
+    assert c["exact"] == c["compared"] == 5 * 3 and c["mismatch"] == 0
+    # a different token at the bottom level of sequence 2, nowhere near an edge: a mismatch, and the walk stops there
+    wrong = {k: v.copy() for k, v in same.items()}
+    a = int(ora["accepted_len"][2, 2])
+    wrong["out_tokens"][2, 2, a] = (int(ora["out_tokens"][2, 2, a]) + 17) % 96
+    margin_before = ora["sample_info"][2, 2, 0]
+    ora["sample_info"][2, 2, 0] = 0.3
+    c = bench.parity_chain(wrong, ora, sample)
+    assert c["mismatch"] == 1 and c["compared"] == 5 * 3 - 2
+    ora["sample_info"][2, 2, 0] = margin_before
+    # an accept decision that flips exactly on its threshold: a tie, the two levels above it are skipped
+    tie = {k: v.copy() for k, v in same.items()}
+    b = 4
+    a = int(ora["accepted_len"][2, b])
+    j = min(a, spec.k[2] - 1)
+    tie["accepted_len"][2, b] = a - 1 if a > 0 else a + 1
+    ora["accept_margin"][2, b, min(int(tie["accepted_len"][2, b]), a)] = 1e-9
+    c = bench.parity_chain(tie, ora, sample)
+    assert c["tie_accept"] == 1 and c["skipped_after_tie"] == 2 and c["mismatch"] == 0
