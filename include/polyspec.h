@@ -346,10 +346,18 @@ polyspec_status polyspec_sharded_chain_handoff(
  *   L_i the acceptance length of the pair (M_i, M_{i+1}) before the insertion, L_{i-new} that of
  *   (M_i, M_new) and L_new that of (M_new, M_{i+1}) after it.  Writes both sides (either pointer may be
  *   NULL) and returns 1 if the condition holds, 0 if not, -1 on non-positive inputs.
+ * polyspec_cost_insertion_drafter -- Theorem 3.2, second condition, as its proof derives it (the three-model
+ *   case, M_new between M_i and the drafter M_{i+1}): the insertion also pays off if
+ *     T_new / T_{i+1}  <  beta (L_new / L_i - 1),
+ *   the sign of the last two terms of the difference of the two Lemma 3.1 totals; L_new and L_i as above,
+ *   T_{i+1} the drafter's forward-pass cost, beta its scaling factor (Lemma 3.1).  The theorem's statement
+ *   prints other subscripts for this condition; the proof's are used.  Same outputs and return values.
  */
 double polyspec_cost_total_time(int n, const double* T /* host [n] */, const double* L /* host [n-1] */, double beta, double N);
 int polyspec_cost_insertion(double T_new, double T_i, double L_new, double L_i, double L_i_new,
                             double* lhs /* host out */, double* rhs /* host out */);
+int polyspec_cost_insertion_drafter(double T_new, double T_next, double L_new, double L_i, double beta,
+                                    double* lhs /* host out */, double* rhs /* host out */);
 
 /*
  * Staged verification with a threshold (Section 3.3, "Staged Verification"; Algorithm 1, three models)

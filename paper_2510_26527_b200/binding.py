@@ -31,7 +31,7 @@ EXPORTS = (
     "polyspec_verify_from_hidden_workspace", "polyspec_verify_from_hidden", "polyspec_lm_head",
     "polyspec_from_hidden_project", "polyspec_from_hidden_verify",
     "polyspec_static_scratch_bytes", "polyspec_verify_level_static",
-    "polyspec_cost_total_time", "polyspec_cost_insertion",
+    "polyspec_cost_total_time", "polyspec_cost_insertion", "polyspec_cost_insertion_drafter",
     "polyspec_sharded_level_sizes", "polyspec_sharded_level_stats", "polyspec_sharded_level_decide",
     "polyspec_sharded_level_pick",
     "polyspec_sharded_chain_sizes", "polyspec_sharded_chain_stats", "polyspec_sharded_chain_gather",
@@ -126,6 +126,8 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_cost_total_time.argtypes = [ci, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), ctypes.c_double, ctypes.c_double]
     lib.polyspec_cost_insertion.restype = ci
     lib.polyspec_cost_insertion.argtypes = [ctypes.c_double] * 5 + [ctypes.POINTER(ctypes.c_double)] * 2
+    lib.polyspec_cost_insertion_drafter.restype = ci
+    lib.polyspec_cost_insertion_drafter.argtypes = [ctypes.c_double] * 5 + [ctypes.POINTER(ctypes.c_double)] * 2
     lib.polyspec_static_scratch_bytes.restype = sz
     lib.polyspec_static_scratch_bytes.argtypes = []
     lib.polyspec_verify_level_static.restype = ci
@@ -597,6 +599,16 @@ def polyspec_cost_insertion(T_new: float, T_i: float, L_new: float, L_i: float, 
     lhs, rhs = ctypes.c_double(0.0), ctypes.c_double(0.0)
     r = load_library().polyspec_cost_insertion(float(T_new), float(T_i), float(L_new), float(L_i), float(L_i_new),
                                                ctypes.byref(lhs), ctypes.byref(rhs))
+    if r < 0:
+        raise ValueError("all five quantities must be positive")
+    return bool(r), lhs.value, rhs.value
+
+
+def polyspec_cost_insertion_drafter(T_new: float, T_next: float, L_new: float, L_i: float, beta: float):
+    """Theorem 3.2, second condition (as its proof derives it): (improves, T_new / T_{i+1}, beta (L_new / L_i - 1))."""
+    lhs, rhs = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    r = load_library().polyspec_cost_insertion_drafter(float(T_new), float(T_next), float(L_new), float(L_i), float(beta),
+                                                       ctypes.byref(lhs), ctypes.byref(rhs))
     if r < 0:
         raise ValueError("all five quantities must be positive")
     return bool(r), lhs.value, rhs.value

@@ -386,6 +386,16 @@ int polyspec_cost_insertion(double T_new, double T_i, double L_new, double L_i, 
     return a < b ? 1 : 0;
 }
 
+int polyspec_cost_insertion_drafter(double T_new, double T_next, double L_new, double L_i, double beta, double* lhs, double* rhs)
+{
+    if (!(T_next > 0.0) || !(T_new > 0.0) || !(L_new > 0.0) || !(L_i > 0.0) || !(beta > 0.0)) return -1;
+    const double a = T_new / T_next;
+    const double b = beta * (L_new / L_i - 1.0);
+    if (lhs) *lhs = a;
+    if (rhs) *rhs = b;
+    return a < b ? 1 : 0;
+}
+
 // ---- greedy matching: only the verifiers' rows are read (arg max), the drafter contributes its tokens
 namespace {
 polyspec_status greedy_shape(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt, long long* total_rows)

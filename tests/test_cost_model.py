@@ -54,3 +54,53 @@ def test_total_time_matches_the_dualistic_formula_and_the_restatement(lib):
     assert np.isnan(binding.polyspec_cost_total_time([1.0, 2.0], [0.0], 1.0, 10))
     with pytest.raises(ValueError):
         binding.polyspec_cost_insertion(1.0, 0.0, 1.0, 1.0, 1.0)
+
+
+def test_both_insertion_conditions_are_the_proofs_partial_sums_of_the_time_difference(lib):
+    """Proof of Theorem 3.2, three-model case: (time with M_new) - (time without) is a sum of three terms, the first
+    condition says the first two sum to less than zero, the second that the last two do.  The difference itself is
+    taken from Lemma 3.1's totals (pinned above), the terms are isolated by switching costs off: with T_{i+1} = 0 the
+    difference is the first two terms, with T_i = 0 the last two.  Under the proof's ordering L_{i-new} > L_new > L_i
+    either condition then implies that the insertion lowers the total."""
+    r = np.random.default_rng(7)
+    seen = {(a, b): 0 for a in (False, True) for b in (False, True)}
+    for _ in range(4000):
+        N = 1000.0
+        T_i, T_next = r.uniform(5, 60), r.uniform(0.5, 15)
+        T_new = r.uniform(0.2, 1.0) * T_i
+        L_i = r.uniform(1.5, 5)
+        L_new = L_i * r.uniform(0.7, 2.2)
+        L_i_new = L_new * r.uniform(0.8, 1.8)
+        beta = r.uniform(0.5, 6)
+
+        def diff(t_i, t_next):
+            with_new = cost_model.total_time([t_i, T_new, t_next], [L_i_new, L_new], beta, N)
+            without = cost_model.total_time([t_i, t_next], [L_i], beta, N)
+            return with_new - without
+
+        l1, r1 = cost_model.insertion_sides(T_new, T_i, L_new, L_i, L_i_new)
+        l2, r2 = cost_model.insertion_sides_drafter(T_new, T_next, L_new, L_i, beta)
+        first_two, last_two = diff(T_i, 0.0), diff(0.0, T_next)
+        if abs(l1 - r1) > 1e-9:
+            assert (l1 < r1) == (first_two < 0)
+        if abs(l2 - r2) > 1e-9:
+            assert (l2 < r2) == (last_two < 0)
+        # the three terms: first_two + last_two counts the middle one (N / L_new T_new) twice
+        assert diff(T_i, T_next) == pytest.approx(first_two + last_two - N / L_new * T_new, rel=1e-9, abs=1e-6)
+        if L_i_new > L_new > L_i and (l1 < r1 or l2 < r2):
+            assert diff(T_i, T_next) < 0
+        seen[(l1 < r1, l2 < r2)] += 1
+        got, g_l, g_r = binding.polyspec_cost_insertion_drafter(T_new, T_next, L_new, L_i, beta)
+        assert got == (l2 < r2) and g_l == pytest.approx(l2, rel=1e-15) and g_r == pytest.approx(r2, rel=1e-14, abs=1e-15)
+    assert all(v > 20 for v in seen.values()), seen                  # every combination of the two conditions occurred
+    with pytest.raises(ValueError):
+        binding.polyspec_cost_insertion_drafter(1.0, 1.0, 1.0, 1.0, 0.0)
+
+
+def test_second_condition_on_the_rows_of_table_1(lib):
+    """Table 1 prints no value for the second condition and no beta; with beta = 1 the drafter-side condition fails in all
+    three rows (T_new exceeds T_{i+1} in each), so the printed verdicts rest on the first condition alone."""
+    for name, T_i, L_i_new, T_new, L_new, T_next, L_i, p_lhs, p_rhs, improves in _rows():
+        ok, lhs, rhs = binding.polyspec_cost_insertion_drafter(T_new, T_next, L_new, L_i, 1.0)
+        assert lhs == pytest.approx(T_new / T_next) and lhs > 1.0 and not ok
+        assert (rhs < 0) == (L_new < L_i)
