@@ -40,7 +40,8 @@ inline bool aligned16s(const void* p) { return (reinterpret_cast<uintptr_t>(p) &
 __host__ __device__ inline size_t stats_part_bytes(long long rows) { return static_cast<size_t>(rows) * 12; }
 __host__ __device__ inline size_t gather_part_bytes(int B, int slots) { return static_cast<size_t>(B) * slots * 8; }
 // Mass record: double mass[B] (what the slice holds of the distribution being sampled), double pmass[B]
-// (what it holds of P at the same row, filled in when it holds nothing of the residual: needed if no rank does).
+// (what it holds of P at the same row, filled in when it holds nothing of the residual: needed if no rank does);
+// both carry the row's common factor Z_p (see resid()), the same on every rank, which the search never needs.
 __host__ __device__ inline size_t mass_record_bytes(int B) { return (static_cast<size_t>(B) * 16 + 255) / 256 * 256; }
 
 // What `decide` leaves for `pick`, per sequence.
@@ -245,9 +246,8 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) shard
     const void* prow = static_cast<const char*>(p.logits_p) + (static_cast<size_t>(b) * p.rows_p + a) * row_bytes;
     const void* qrow = static_cast<const char*>(p.logits_q) + (static_cast<size_t>(b) * p.rows_q + (use_q ? a : 0)) * row_bytes;
     const int ntiles = (p.V_local + kTile - 1) / kTile;
-    const float iZp = static_cast<float>(1.0 / sp.Z);
-    const float iZq = use_q ? static_cast<float>(1.0 / sq.Z) : 0.0f;
-    tiles_pass<DT>(prow, qrow, p.V_local, p.c, sp.E, iZp, sq.E, iZq, use_q, tile_sum, 0, ntiles);
+    const RowScale sc = row_scale(sp.E, sp.Z, sq.E, sq.Z, use_q);
+    tiles_pass<DT>(prow, qrow, p.V_local, p.c, sc, use_q, tile_sum, 0, ntiles);
     __syncthreads();
     int t0, t1;
     double mine, incl;
@@ -261,7 +261,7 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) shard
     const bool no_mass = use_q && !(sh_share > 0.0);
     if (no_mass) {
         __syncthreads();
-        tiles_pass<DT>(prow, qrow, p.V_local, p.c, sp.E, iZp, sq.E, 0.0f, false, tile_sum, 0, ntiles);
+        tiles_pass<DT>(prow, qrow, p.V_local, p.c, sc, false, tile_sum, 0, ntiles);
         __syncthreads();
         if (tid < 32) {
             const double pshare = share_of_tiles(tile_sum, ntiles, lane, &t0, &t1, &mine, &incl);
@@ -302,8 +302,7 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) shard
     bool use_q = dec.use_q != 0;
     const void* prow = static_cast<const char*>(p.logits_p) + (static_cast<size_t>(b) * p.rows_p + dec.a) * row_bytes;
     const void* qrow = static_cast<const char*>(p.logits_q) + (static_cast<size_t>(b) * p.rows_q + (use_q ? dec.a : 0)) * row_bytes;
-    const float iZp = static_cast<float>(1.0 / dec.Zp);
-    const float iZq = use_q ? static_cast<float>(1.0 / dec.Zq) : 0.0f;
+    const RowScale sc = row_scale(dec.Ep, dec.Zp, dec.Eq, dec.Zq, use_q);
 
     // the residual vanished in floating point on every rank: sample P instead (its masses are in the records too)
     if (tid == 0) {
@@ -340,7 +339,7 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) shard
             int t0, t1;
             double mine, incl;
             (void)share_of_tiles(tile_sum, ntiles, lane, &t0, &t1, &mine, &incl);
-            token = pick_in_share<DT>(prow, qrow, p.V_local, p.c, dec.Ep, iZp, dec.Eq, iZq, use_q, tile_sum, t0, t1, mine, incl,
+            token = pick_in_share<DT>(prow, qrow, p.V_local, p.c, sc, use_q, tile_sum, t0, t1, mine, incl,
                                       base, target, lane);
             if (token >= 0) token += p.rank * p.V_local;
         }

@@ -140,14 +140,31 @@ __device__ __forceinline__ RowStat merge_partials(const float2* part, int parts,
 
 __device__ __forceinline__ bool stat_ok(const RowStat& s) { return s.Z > 0.0 && s.Z < 1.0e300; }   // false for NaN too
 
-// The residual (or, without q, the probability) of one element, in a fixed operation order
-// so that the sum pass and the rescan produce identical values.
-__device__ __forceinline__ float resid(float zp, float zq, float c, float Ep, float iZp, float Eq, float iZq, bool use_q)
+// The residual (or, without q, the probability) of one element, up to the row's common factor: with
+// a = 2^(z_p c - E_p) = P Z_p and b = 2^(z_q c - E_q) = Q Z_q the value is max(0, a - rho b) = Z_p max(0, P - Q) for
+// rho = Z_p / Z_q.  The inverse-CDF search only ever compares partial sums with u times the total, so the factor
+// Z_p never has to be divided out.  One fixed operation order, so that the sum pass and the rescan produce
+// identical values.
+template <bool USE_Q>
+__device__ __forceinline__ float resid(float zp, float zq, float c, float nEp, float nEq, float nrho)
 {
-    const float pv = __fmul_rn(ex2f(__fmaf_rn(zp, c, -Ep)), iZp);
-    if (!use_q) return pv;
-    const float qv = __fmul_rn(ex2f(__fmaf_rn(zq, c, -Eq)), iZq);
-    return fmaxf(0.0f, __fsub_rn(pv, qv));
+    const float a = ex2f(__fmaf_rn(zp, c, nEp));
+    if (!USE_Q) return a;
+    const float b = ex2f(__fmaf_rn(zq, c, nEq));
+    return fmaxf(0.0f, __fmaf_rn(nrho, b, a));
+}
+
+// The per-row constants of resid(): the negated references and the negated ratio of the normalisers.
+struct RowScale {
+    float nEp, nEq, nrho;
+};
+__device__ __forceinline__ RowScale row_scale(float Ep, double Zp, float Eq, double Zq, bool use_q)
+{
+    RowScale s;
+    s.nEp = -Ep;
+    s.nEq = -Eq;
+    s.nrho = use_q ? -static_cast<float>(Zp / Zq) : 0.0f;
+    return s;
 }
 
 __device__ __forceinline__ float sum8(const float* r)
@@ -156,20 +173,26 @@ __device__ __forceinline__ float sum8(const float* r)
                      __fadd_rn(__fadd_rn(r[4], r[5]), __fadd_rn(r[6], r[7])));
 }
 
-template <int DT>
-__device__ __forceinline__ void tile_resid(const void* prow, const void* qrow, int v, int V, float c,
-                                           float Ep, float iZp, float Eq, float iZq, bool use_q, float* r)
+template <int DT, bool USE_Q>
+__device__ __forceinline__ void tile_resid_q(const void* prow, const void* qrow, int v, int V, float c, const RowScale sc, float* r)
 {
     if (v < V) {
         float zp[8], zq[8];
         load8<DT>(prow, v, zp);
-        if (use_q) load8<DT>(qrow, v, zq);
+        if (USE_Q) load8<DT>(qrow, v, zq);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) r[e] = resid(zp[e], use_q ? zq[e] : 0.0f, c, Ep, iZp, Eq, iZq, use_q);
+        for (int e = 0; e < 8; ++e) r[e] = resid<USE_Q>(zp[e], USE_Q ? zq[e] : 0.0f, c, sc.nEp, sc.nEq, sc.nrho);
     } else {
 #pragma unroll
         for (int e = 0; e < 8; ++e) r[e] = 0.0f;
     }
+}
+template <int DT>
+__device__ __forceinline__ void tile_resid(const void* prow, const void* qrow, int v, int V, float c, const RowScale sc, bool use_q,
+                                           float* r)
+{
+    if (use_q) tile_resid_q<DT, true>(prow, qrow, v, V, c, sc, r);
+    else tile_resid_q<DT, false>(prow, qrow, v, V, c, sc, r);
 }
 
 __device__ __forceinline__ double warp_incl_scan(double x, int lane)
@@ -212,56 +235,94 @@ __device__ __forceinline__ void cluster_barrier(const ClusterCtx& cl)
     }
 }
 
+// The sum of one lane's eight elements of a tile, added as a fixed tree.
+template <int DT, bool USE_Q>
+__device__ __forceinline__ float lane_sum(const RawTile<DT>& rp, const RawTile<DT>& rq, float c, const RowScale sc)
+{
+    float zp[8], zq[8], r[8];
+    rp.unpack(zp);
+    if (USE_Q) rq.unpack(zq);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) r[e] = resid<USE_Q>(zp[e], USE_Q ? zq[e] : 0.0f, c, sc.nEp, sc.nEq, sc.nrho);
+    return sum8(r);
+}
+
+// Tiles handled together by one warp in the row pass: their four per-lane sums are reduced over the warp in one
+// transposed butterfly (6 shuffles for four tiles instead of 20).
+constexpr int kTileGroup = 4;
+
+// x0..x3 are a lane's sums of four tiles.  Returns, in the lanes with (lane >> 3) == i, the sum of x_i over the warp,
+// added in the order of a plain xor-butterfly (16, 8, 4, 2, 1), so a tile's sum does not depend on whether it was
+// reduced alone or in a group.
+__device__ __forceinline__ float reduce_four_tiles(float x0, float x1, float x2, float x3, int lane)
+{
+    const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
+    float k0 = up16 ? x2 : x0, k1 = up16 ? x3 : x1;
+    const float g0 = up16 ? x0 : x2, g1 = up16 ? x1 : x3;
+    k0 = __fadd_rn(k0, __shfl_xor_sync(0xffffffffu, g0, 16));
+    k1 = __fadd_rn(k1, __shfl_xor_sync(0xffffffffu, g1, 16));
+    float k = up8 ? k1 : k0;
+    const float g = up8 ? k0 : k1;
+    k = __fadd_rn(k, __shfl_xor_sync(0xffffffffu, g, 8));
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) k = __fadd_rn(k, __shfl_xor_sync(0xffffffffu, k, o));
+    return k;
+}
+
 // The sums of the residual (or of P) over tiles [tlo, thi) of one row, one float per tile in tile_sum[t]; all warps
-// of the CTA take part, no synchronisation inside.
-template <int DT>
-__device__ __forceinline__ void tiles_pass(const void* prow, const void* qrow, int V, float c, float Ep, float iZp, float Eq, float iZq,
-                                           bool use_q, float* tile_sum, int tlo, int thi)
+// of the CTA take part, no synchronisation inside.  Whole tiles go in groups of four per warp while there are
+// enough groups to occupy every warp; what is left (and the ragged last tile) goes one tile per warp.
+template <int DT, bool USE_Q>
+__device__ __forceinline__ void tiles_pass_q(const void* prow, const void* qrow, int V, float c, const RowScale sc, float* tile_sum,
+                                             int tlo, int thi)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    // kUnroll tiles per warp and step: all their loads are issued before the first is used, so a warp
-    // has kUnroll (x2 with q) 16-byte loads per lane in flight instead of one.  Each tile's sum is
-    // computed exactly as in the rescan below, whatever the grouping.
-    constexpr int kUnroll = Unroll<DT>::value;
-    for (int t0 = tlo + warp * kUnroll; t0 < thi; t0 += kWalkWarps * kUnroll) {
-        RawTile<DT> rp[kUnroll], rq[kUnroll];
+    const int whole = min(thi, V / kTile);              // tiles below this index lie wholly inside the row
+    int ngroups = (whole - tlo) / kTileGroup;
+    if (ngroups < kWalkWarps) ngroups = 0;
+    for (int g = warp; g < ngroups; g += kWalkWarps) {
+        const int t0 = tlo + g * kTileGroup;
+        float x[kTileGroup];
+        // tiles whose loads are in flight together per lane: two of 2-byte logits (four 16-byte vectors with q),
+        // one of float32 (the same four vectors)
+        constexpr int kFly = (DT == POLYSPEC_BF16) ? 2 : 1;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int v = (t0 + u) * kTile + lane * 8;
-            if (v < V) {
-                rp[u].load(prow, v);
-                if (use_q) rq[u].load(qrow, v);
+        for (int h = 0; h < kTileGroup; h += kFly) {
+            RawTile<DT> rp[kFly], rq[kFly];
+#pragma unroll
+            for (int f = 0; f < kFly; ++f) {
+                const int v = (t0 + h + f) * kTile + lane * 8;
+                rp[f].load(prow, v);
+                if (USE_Q) rq[f].load(qrow, v);
             }
+#pragma unroll
+            for (int f = 0; f < kFly; ++f) x[h + f] = lane_sum<DT, USE_Q>(rp[f], rq[f], c, sc);
         }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            if (t0 + u < thi) {                     // warp-uniform
-                const int v = (t0 + u) * kTile + lane * 8;
-                float r[8];
-                if (v < V) {
-                    float zp[8], zq[8];
-                    rp[u].unpack(zp);
-                    if (use_q) rq[u].unpack(zq);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) r[e] = resid(zp[e], use_q ? zq[e] : 0.0f, c, Ep, iZp, Eq, iZq, use_q);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) r[e] = 0.0f;
-                }
-                float x = sum8(r);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
-                if (lane == 0) tile_sum[t0 + u] = x;
-            }
-        }
+        const float k = reduce_four_tiles(x[0], x[1], x[2], x[3], lane);
+        if ((lane & 7) == 0) tile_sum[t0 + (lane >> 3)] = k;
     }
+    for (int t = tlo + ngroups * kTileGroup + warp; t < thi; t += kWalkWarps) {
+        float r[8];
+        tile_resid_q<DT, USE_Q>(prow, qrow, t * kTile + lane * 8, V, c, sc, r);
+        float x = sum8(r);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
+        if (lane == 0) tile_sum[t] = x;
+    }
+}
+template <int DT>
+__device__ __forceinline__ void tiles_pass(const void* prow, const void* qrow, int V, float c, const RowScale sc, bool use_q,
+                                           float* tile_sum, int tlo, int thi)
+{
+    if (use_q) tiles_pass_q<DT, true>(prow, qrow, V, c, sc, tile_sum, tlo, thi);
+    else tiles_pass_q<DT, false>(prow, qrow, V, c, sc, tile_sum, tlo, thi);
 }
 
 // The token at `target` of the row's running sum, for the warp of the share that contains it: lane i of the warp
 // owns tiles [t0, t1) of the share with sum `mine` and inclusive running sum `incl` over the lanes, `base` is the mass
 // before the share.  Returns the token in every lane (-1 if the share holds no mass).
 template <int DT, bool COHERENT = false>
-__device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow, int V, float c, float Ep, float iZp, float Eq, float iZq,
+__device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow, int V, float c, const RowScale sc,
                                              bool use_q, const float* tile_sum, int t0, int t1, double mine, double incl,
                                              double base, double target, int lane)
 {
@@ -295,7 +356,7 @@ __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow,
     }
     if (tile >= 0) {
         float r[8];
-        tile_resid<DT>(prow, qrow, tile * kTile + lane * 8, V, c, Ep, iZp, Eq, iZq, use_q, r);
+        tile_resid<DT>(prow, qrow, tile * kTile + lane * 8, V, c, sc, use_q, r);
         double lane_sum = 0.0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) lane_sum += static_cast<double>(r[e]);
@@ -324,7 +385,8 @@ __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow,
 }
 
 // Inverse CDF of the residual (use_q) or of P (bonus / fallback) at uniform u.
-// Returns the token (same value in every thread) and the total mass through *total_out.
+// Returns the token (same value in every thread) and, through *total_out, the total mass times the row's
+// common factor Z_p (only its sign is meaningful to the caller).
 template <int DT>
 __device__ int sample_row(const void* prow, const void* qrow, int V, float c, RowStat sp, RowStat sq, bool use_q,
                           float u, float* tile_sum, SampleShared* sh, double* total_out, const ClusterCtx cl)
@@ -334,11 +396,9 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
     // this CTA's share of the row: tiles [tlo, thi)
     const int tiles_per_rank = (ntiles + cl.size - 1) / cl.size;
     const int tlo = min(cl.rank * tiles_per_rank, ntiles), thi = min(tlo + tiles_per_rank, ntiles);
-    const float iZp = static_cast<float>(1.0 / sp.Z);
-    const float iZq = use_q ? static_cast<float>(1.0 / sq.Z) : 0.0f;
-    const float Ep = sp.E, Eq = sq.E;
+    const RowScale sc = row_scale(sp.E, sp.Z, sq.E, sq.Z, use_q);
 
-    tiles_pass<DT>(prow, qrow, V, c, Ep, iZp, Eq, iZq, use_q, tile_sum, tlo, thi);
+    tiles_pass<DT>(prow, qrow, V, c, sc, use_q, tile_sum, tlo, thi);
     __syncthreads();
 
     // each lane of warp 0 owns a contiguous run of the CTA's tiles; tile sums are added in double, in order
@@ -373,7 +433,7 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
         if (owner_rank < 0) { owner_rank = last_mass; base = last_base; }      // u not below 1, or rounding
         int token = -1;
         if (owner_rank == cl.rank) {
-            token = pick_in_share<DT>(prow, qrow, V, c, Ep, iZp, Eq, iZq, use_q, tile_sum, t0, t1, mine, incl, base, target, lane);
+            token = pick_in_share<DT>(prow, qrow, V, c, sc, use_q, tile_sum, t0, t1, mine, incl, base, target, lane);
         }
         if (lane == 0) sh->total = total;
         // the CTA that holds the token tells every CTA (with no mass anywhere, CTA 0 reports -1)
