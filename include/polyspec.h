@@ -116,13 +116,6 @@ polyspec_status polyspec_verify_level(
  *   accepted_len, block_len, out_len   out [n_models-1, B]; out_len = accepted_len + 1
  *   out_tokens    out [n_models-1, B, kmax+1]: stream emitted by each level, -1 past out_len;
  *                 level 0's stream is the committed output
- *
- * polyspec_verify_chain_launches -- how many kernels such a call (or a polyspec_verify_level call with
- *   n_models = 2) enqueues: 2 in general (row statistics, then decision and sampling); 1 for a small batch
- *   (the paper's setting is batch size 1, Section 4.1) whose rows fit the shared memory of one eight-CTA
- *   cluster per sequence (B <= 16 and, per sequence, about 1.8 MB of logits), which then does both steps
- *   without reading a logit from global memory twice.  The results do not depend on which of the two ran.
- *   Host arithmetic only; the answer assumes a device that can place such a cluster (a B200 can).
  */
 typedef struct {
     const void* logits;   /* device pointer, [B, rows, V] */
@@ -131,8 +124,6 @@ typedef struct {
 
 polyspec_status polyspec_verify_chain_workspace(int n_models, const int* k /* host */, const int* rows /* host [n_models] */,
                                                 int B, int V, polyspec_dtype dt, size_t* bytes /* host out */);
-polyspec_status polyspec_verify_chain_launches(int n_models, const int* k /* host */, const int* rows /* host [n_models] */,
-                                              int B, int V, polyspec_dtype dt, int* launches /* host out */);
 polyspec_status polyspec_verify_chain(
     const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */,
     const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,

@@ -24,7 +24,7 @@ MAX_K, MAX_MODELS = 32, 8
 EXPORTS = (
     "polyspec_status_string", "polyspec_version", "polyspec_last_cuda_error",
     "polyspec_verify_level_workspace", "polyspec_verify_level",
-    "polyspec_verify_chain_workspace", "polyspec_verify_chain", "polyspec_verify_chain_launches",
+    "polyspec_verify_chain_workspace", "polyspec_verify_chain",
     "polyspec_chain_row_stats", "polyspec_chain_walk",
     "polyspec_verify_chain_greedy_workspace", "polyspec_verify_chain_greedy",
     "polyspec_verify_chain_host_workspace", "polyspec_verify_chain_host",
@@ -92,8 +92,6 @@ def load_library() -> ctypes.CDLL:
                                           i32p, i32p, f32p, f32p, i32p, vp, sz, vp]
     lib.polyspec_verify_chain_workspace.restype = ci
     lib.polyspec_verify_chain_workspace.argtypes = [ci, cip, cip, ci, ci, ci, szp]
-    lib.polyspec_verify_chain_launches.restype = ci
-    lib.polyspec_verify_chain_launches.argtypes = [ci, cip, cip, ci, ci, ci, cip]
     lib.polyspec_verify_chain.restype = ci
     lib.polyspec_verify_chain.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, i32p, f32p, ci, ci, ci, cf,
                                           i32p, i32p, i32p, i32p, i32p, vp, sz, vp]
@@ -266,14 +264,6 @@ def polyspec_verify_chain_workspace(k: Sequence[int], rows: Sequence[int], B: in
     return n.value
 
 
-def polyspec_verify_chain_launches(k: Sequence[int], rows: Sequence[int], B: int, V: int, dt: int) -> int:
-    """Kernels a polyspec_verify_chain call of this shape enqueues: 1 (small batch, one cluster kernel) or 2."""
-    n = ctypes.c_int(0)
-    _check(load_library().polyspec_verify_chain_launches(len(rows), _int_array(k), _int_array(rows), B, V, dt, ctypes.byref(n)),
-           "polyspec_verify_chain_launches")
-    return n.value
-
-
 def chain_outputs(L: int, B: int, kmax: int, device, pin=False) -> dict:
     kw = {"dtype": torch.int32, "device": device}
     if pin:
@@ -384,7 +374,6 @@ class ChainCall:
         self._arr = (ModelLogits * self.n)(*[ModelLogits(m.data_ptr(), r) for m, r in zip(models, self.rows)])
         self._k = _int_array(self.k)
         self.stream = stream
-        self.launches = polyspec_verify_chain_launches(self.k, self.rows, self.B, self.V, self.dt)   # kernels launch() enqueues
 
     def _tail(self):
         o = self.out

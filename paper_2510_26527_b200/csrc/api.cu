@@ -178,24 +178,8 @@ polyspec_status run_chain_two_launch(const ChainArgs& a)
     return run_walk(a);
 }
 
-// One launch when the problem is small enough for the cluster kernel, else the two launches; the same results.
 polyspec_status run_chain(const ChainArgs& a)
 {
-    if (!a.draft_tokens || !a.uniforms || !a.accepted_len) return POLYSPEC_ERR_INVALID_ARG;
-    if (a.parts_override == 0 && a.spin_limit == 0 && a.B <= kSmallMaxBatch) {
-        StatsPlan pl;
-        StatsParams sp;
-        polyspec_status st = prepare_chain(a, &pl, &sp);
-        if (st != POLYSPEC_OK) return st;
-        SmallChainPlan small;
-        if (small_chain_plan(sp.t, a.B, a.V, a.dt, pl, &small)) {
-            WalkParams wp;
-            fill_walk_params(a, sp, pl.parts, &wp);
-            bool launched = false;
-            if (cuda_failed(launch_small_chain(a.dt, wp, small, a.stream, &launched))) return POLYSPEC_ERR_CUDA;
-            if (launched) return POLYSPEC_OK;
-        }
-    }
     return run_chain_two_launch(a);
 }
 
@@ -326,21 +310,6 @@ polyspec_status polyspec_verify_chain_workspace(int n_models, const int* k, cons
     polyspec_status st = check_chain_shape(n_models, k, rows, B, V, dt, &total);
     if (st != POLYSPEC_OK) return st;
     *bytes = chain_workspace_bytes(total, n_models, B, V, dt);
-    return POLYSPEC_OK;
-}
-
-polyspec_status polyspec_verify_chain_launches(int n_models, const int* k, const int* rows, int B, int V, polyspec_dtype dt,
-                                              int* launches)
-{
-    if (!launches) return POLYSPEC_ERR_INVALID_ARG;
-    long long total = 0;
-    polyspec_status st = check_chain_shape(n_models, k, rows, B, V, dt, &total);
-    if (st != POLYSPEC_OK) return st;
-    RowTable t;
-    const void* none[kMaxModels] = {};
-    if (fill_rows(t, none, rows, n_models, B) < 0) return POLYSPEC_ERR_UNSUPPORTED;
-    SmallChainPlan small;
-    *launches = (B <= kSmallMaxBatch && small_chain_plan(t, B, V, dt, plan_stats(total, V, dt), &small)) ? 1 : 2;
     return POLYSPEC_OK;
 }
 

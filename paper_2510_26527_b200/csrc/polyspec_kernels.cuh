@@ -92,21 +92,6 @@ cudaError_t launch_walk(polyspec_dtype dt, const WalkParams& p, cudaStream_t str
 // Greedy matching: reads arg-max partials (launch_stats with argmax = true) of the verifiers' rows only.
 cudaError_t launch_greedy_walk(const WalkParams& p, cudaStream_t stream);
 
-// Small batches in one launch (small_kernel.cu): a cluster of eight CTAs per sequence stages all of the sequence's
-// rows in shared memory, computes the partials there and runs the level loop on them.  small_chain_plan says
-// whether a problem qualifies (few sequences, rows that fit, the segment length of small problems) and how it is
-// laid out; launch_small_chain sets *launched to false, and launches nothing, on a device that cannot place such
-// a cluster.  Results are those of launch_stats followed by launch_walk.
-constexpr int kSmallMaxBatch = 16;
-struct SmallChainPlan {
-    int tiles_per_rank;
-    int slice_bytes;
-    int rows_per_seq;
-    size_t smem_bytes;
-};
-bool small_chain_plan(const RowTable& t, int B, int V, polyspec_dtype dt, const StatsPlan& pl, SmallChainPlan* out);
-cudaError_t launch_small_chain(polyspec_dtype dt, const WalkParams& w, const SmallChainPlan& plan, cudaStream_t stream, bool* launched);
-
 // The level call as two launches on a workspace that holds the partials only (api.cu); polyspec_verify_level_static
 // runs it on the library's built-in scratch.
 polyspec_status verify_level_two_launch_workspace(int B, int k, int V, polyspec_dtype dt, size_t* bytes);

@@ -113,8 +113,10 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
         uint32_t bytes;
         item_span<DT>(p, item, &src, &bytes);
 
-        SoftmaxAcc<DT> acc;
-        acc.init();
+        float E = kEmptyRef;
+        float s[kVecPerLane];
+#pragma unroll
+        for (int u = 0; u < kVecPerLane; ++u) s[u] = 0.0f;
         // arg-max state of this lane: its elements come in ascending index order, so a strictly
         // larger value is always the first occurrence among the lane's own
         float best = -INFINITY;
@@ -144,11 +146,24 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
                 const int idx = lane + u * 32;
                 r[u] = (idx < nvec) ? ld_shared_v4(base + idx * 16) : EL::neg_inf();
             }
+            float z[kVecPerLane][EPV];
             if (MODE == 0) {
-                acc.add_chunk(r, c);
+                const float M = EL::vec_max(r);
+#pragma unroll
+                for (int u = 0; u < kVecPerLane; ++u) EL::unpack(r[u], z[u]);
+                const float En = (M == -INFINITY) ? kEmptyRef : ceilf(M * c);
+                if (En > E) {
+                    const float sc = pow2_neg(E - En);
+#pragma unroll
+                    for (int u = 0; u < kVecPerLane; ++u) s[u] *= sc;
+                    E = En;
+                }
+#pragma unroll
+                for (int u = 0; u < kVecPerLane; ++u)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) s[u] += ex2f(__fmaf_rn(z[u][e], c, -E));
             } else {
                 constexpr int ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
-                float z[kVecPerLane][EPV];
 #pragma unroll
                 for (int u = 0; u < kVecPerLane; ++u) {
                     EL::unpack(r[u], z[u]);
@@ -184,8 +199,14 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
             continue;
         }
 
-        const float2 part = acc.finish();
-        if (lane == 0) p.partials[item] = part;
+        // lanes -> warp: rebase every lane to the warp's largest reference (exact), then add
+        float Ew = E;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) Ew = fmaxf(Ew, __shfl_xor_sync(0xffffffffu, Ew, o));
+        float sw = ((s[0] + s[1]) + (s[2] + s[3])) * pow2_neg(E - Ew);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(0xffffffffu, sw, o);
+        if (lane == 0) p.partials[item] = make_float2(Ew, sw);
     }
 }
 

@@ -138,51 +138,5 @@ template <> struct Elems<POLYSPEC_F32> {
     }
 };
 
-// The online softmax-normaliser pair of one lane over a row segment that arrives in 2 KiB chunks (four 16-byte
-// vectors per lane and chunk): sum 2^(z c - E) = s[0] + s[1] + s[2] + s[3], E an integer-valued reference at or
-// just above the running maximum of z c.  One definition for every kernel that produces partials, so that a
-// segment's partial has the same bits wherever it was computed.
-template <int DT> struct SoftmaxAcc {
-    using EL = Elems<DT>;
-    float E;
-    float s[kVecPerLane];
-    __device__ __forceinline__ void init()
-    {
-        E = kEmptyRef;
-#pragma unroll
-        for (int u = 0; u < kVecPerLane; ++u) s[u] = 0.0f;
-    }
-    // r: the lane's vectors of this chunk (neg_inf() where the chunk has none for it)
-    __device__ __forceinline__ void add_chunk(const uint4 (&r)[kVecPerLane], float c)
-    {
-        float z[kVecPerLane][EL::per_vec];
-        const float M = EL::vec_max(r);
-#pragma unroll
-        for (int u = 0; u < kVecPerLane; ++u) EL::unpack(r[u], z[u]);
-        const float En = (M == -INFINITY) ? kEmptyRef : ceilf(M * c);
-        if (En > E) {
-            const float sc = pow2_neg(E - En);
-#pragma unroll
-            for (int u = 0; u < kVecPerLane; ++u) s[u] *= sc;
-            E = En;
-        }
-#pragma unroll
-        for (int u = 0; u < kVecPerLane; ++u)
-#pragma unroll
-            for (int e = 0; e < EL::per_vec; ++e) s[u] += ex2f(__fmaf_rn(z[u][e], c, -E));
-    }
-    // lanes -> warp: rebase every lane to the warp's largest reference (exact), then add; the same pair in every lane
-    __device__ __forceinline__ float2 finish() const
-    {
-        float Ew = E;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) Ew = fmaxf(Ew, __shfl_xor_sync(0xffffffffu, Ew, o));
-        float sw = ((s[0] + s[1]) + (s[2] + s[3])) * pow2_neg(E - Ew);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(0xffffffffu, sw, o);
-        return make_float2(Ew, sw);
-    }
-};
-
 }  // namespace streamdev
 }  // namespace polyspec

@@ -42,26 +42,18 @@ template <int DT> __device__ __forceinline__ float load_logit(const void* row, i
     return static_cast<const float*>(row)[v];
 }
 
-// A 16-byte vector of a row: through the read-only path for rows in global memory; LOCAL rows sit in this CTA's
-// shared memory (the small-batch kernel stages them there) and take a plain load.
-template <bool LOCAL> __device__ __forceinline__ uint4 ld_row(const void* p)
-{
-    if (LOCAL) return *static_cast<const uint4*>(p);
-    return ld_nc(p);
-}
-
 // Eight consecutive logits starting at element v (v a multiple of 8, inside the row).
-template <int DT, bool LOCAL = false> __device__ __forceinline__ void load8(const void* row, int v, float* z)
+template <int DT> __device__ __forceinline__ void load8(const void* row, int v, float* z)
 {
     if (DT == POLYSPEC_BF16) {
-        const uint4 r = ld_row<LOCAL>(static_cast<const unsigned short*>(row) + v);
+        const uint4 r = ld_nc(static_cast<const unsigned short*>(row) + v);
         z[0] = __uint_as_float(r.x << 16); z[1] = __uint_as_float(r.x & 0xffff0000u);
         z[2] = __uint_as_float(r.y << 16); z[3] = __uint_as_float(r.y & 0xffff0000u);
         z[4] = __uint_as_float(r.z << 16); z[5] = __uint_as_float(r.z & 0xffff0000u);
         z[6] = __uint_as_float(r.w << 16); z[7] = __uint_as_float(r.w & 0xffff0000u);
     } else {
-        const uint4 a = ld_row<LOCAL>(static_cast<const float*>(row) + v);
-        const uint4 b = ld_row<LOCAL>(static_cast<const float*>(row) + v + 4);
+        const uint4 a = ld_nc(static_cast<const float*>(row) + v);
+        const uint4 b = ld_nc(static_cast<const float*>(row) + v + 4);
         z[0] = __uint_as_float(a.x); z[1] = __uint_as_float(a.y); z[2] = __uint_as_float(a.z); z[3] = __uint_as_float(a.w);
         z[4] = __uint_as_float(b.x); z[5] = __uint_as_float(b.y); z[6] = __uint_as_float(b.z); z[7] = __uint_as_float(b.w);
     }
@@ -71,10 +63,7 @@ template <int DT, bool LOCAL = false> __device__ __forceinline__ void load8(cons
 template <int DT> struct RawTile;
 template <> struct RawTile<POLYSPEC_BF16> {
     uint4 a;
-    template <bool LOCAL = false> __device__ __forceinline__ void load(const void* row, int v)
-    {
-        a = ld_row<LOCAL>(static_cast<const unsigned short*>(row) + v);
-    }
+    __device__ __forceinline__ void load(const void* row, int v) { a = ld_nc(static_cast<const unsigned short*>(row) + v); }
     __device__ __forceinline__ void unpack(float* z) const
     {
         z[0] = __uint_as_float(a.x << 16); z[1] = __uint_as_float(a.x & 0xffff0000u);
@@ -85,10 +74,10 @@ template <> struct RawTile<POLYSPEC_BF16> {
 };
 template <> struct RawTile<POLYSPEC_F32> {
     uint4 a, b;
-    template <bool LOCAL = false> __device__ __forceinline__ void load(const void* row, int v)
+    __device__ __forceinline__ void load(const void* row, int v)
     {
-        a = ld_row<LOCAL>(static_cast<const float*>(row) + v);
-        b = ld_row<LOCAL>(static_cast<const float*>(row) + v + 4);
+        a = ld_nc(static_cast<const float*>(row) + v);
+        b = ld_nc(static_cast<const float*>(row) + v + 4);
     }
     __device__ __forceinline__ void unpack(float* z) const
     {
@@ -184,13 +173,13 @@ __device__ __forceinline__ float sum8(const float* r)
                      __fadd_rn(__fadd_rn(r[4], r[5]), __fadd_rn(r[6], r[7])));
 }
 
-template <int DT, bool USE_Q, bool LOCAL = false>
+template <int DT, bool USE_Q>
 __device__ __forceinline__ void tile_resid_q(const void* prow, const void* qrow, int v, int V, float c, const RowScale sc, float* r)
 {
     if (v < V) {
         float zp[8], zq[8];
-        load8<DT, LOCAL>(prow, v, zp);
-        if (USE_Q) load8<DT, LOCAL>(qrow, v, zq);
+        load8<DT>(prow, v, zp);
+        if (USE_Q) load8<DT>(qrow, v, zq);
 #pragma unroll
         for (int e = 0; e < 8; ++e) r[e] = resid<USE_Q>(zp[e], USE_Q ? zq[e] : 0.0f, c, sc.nEp, sc.nEq, sc.nrho);
     } else {
@@ -198,12 +187,12 @@ __device__ __forceinline__ void tile_resid_q(const void* prow, const void* qrow,
         for (int e = 0; e < 8; ++e) r[e] = 0.0f;
     }
 }
-template <int DT, bool LOCAL = false>
+template <int DT>
 __device__ __forceinline__ void tile_resid(const void* prow, const void* qrow, int v, int V, float c, const RowScale sc, bool use_q,
                                            float* r)
 {
-    if (use_q) tile_resid_q<DT, true, LOCAL>(prow, qrow, v, V, c, sc, r);
-    else tile_resid_q<DT, false, LOCAL>(prow, qrow, v, V, c, sc, r);
+    if (use_q) tile_resid_q<DT, true>(prow, qrow, v, V, c, sc, r);
+    else tile_resid_q<DT, false>(prow, qrow, v, V, c, sc, r);
 }
 
 __device__ __forceinline__ double warp_incl_scan(double x, int lane)
@@ -225,9 +214,8 @@ struct SampleShared {
 // A sequence may be walked by a cluster of CTAs (small batches: more SMs per sequence).  Every CTA
 // runs the same control flow on the same inputs; only the row pass is divided, by tile ranges.
 struct ClusterCtx {
-    int size;            // CTAs per sequence: 1, 2, 4 or 8
+    int size;       // CTAs per sequence: 1, 2, 4 or 8
     int rank;
-    int tiles_per_rank;  // rank r owns tiles [r * tiles_per_rank, (r + 1) * tiles_per_rank) of every row
 };
 
 __device__ __forceinline__ uint32_t peer_addr(const void* local, int rank)
@@ -284,7 +272,7 @@ __device__ __forceinline__ float reduce_four_tiles(float x0, float x1, float x2,
 // The sums of the residual (or of P) over tiles [tlo, thi) of one row, one float per tile in tile_sum[t]; all warps
 // of the CTA take part, no synchronisation inside.  Whole tiles go in groups of four per warp while there are
 // enough groups to occupy every warp; what is left (and the ragged last tile) goes one tile per warp.
-template <int DT, bool USE_Q, bool LOCAL = false>
+template <int DT, bool USE_Q>
 __device__ __forceinline__ void tiles_pass_q(const void* prow, const void* qrow, int V, float c, const RowScale sc, float* tile_sum,
                                              int tlo, int thi)
 {
@@ -304,8 +292,8 @@ __device__ __forceinline__ void tiles_pass_q(const void* prow, const void* qrow,
 #pragma unroll
             for (int f = 0; f < kFly; ++f) {
                 const int v = (t0 + h + f) * kTile + lane * 8;
-                rp[f].template load<LOCAL>(prow, v);
-                if (USE_Q) rq[f].template load<LOCAL>(qrow, v);
+                rp[f].load(prow, v);
+                if (USE_Q) rq[f].load(qrow, v);
             }
 #pragma unroll
             for (int f = 0; f < kFly; ++f) x[h + f] = lane_sum<DT, USE_Q>(rp[f], rq[f], c, sc);
@@ -315,25 +303,25 @@ __device__ __forceinline__ void tiles_pass_q(const void* prow, const void* qrow,
     }
     for (int t = tlo + ngroups * kTileGroup + warp; t < thi; t += kWalkWarps) {
         float r[8];
-        tile_resid_q<DT, USE_Q, LOCAL>(prow, qrow, t * kTile + lane * 8, V, c, sc, r);
+        tile_resid_q<DT, USE_Q>(prow, qrow, t * kTile + lane * 8, V, c, sc, r);
         float x = sum8(r);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) x = __fadd_rn(x, __shfl_xor_sync(0xffffffffu, x, o));
         if (lane == 0) tile_sum[t] = x;
     }
 }
-template <int DT, bool LOCAL = false>
+template <int DT>
 __device__ __forceinline__ void tiles_pass(const void* prow, const void* qrow, int V, float c, const RowScale sc, bool use_q,
                                            float* tile_sum, int tlo, int thi)
 {
-    if (use_q) tiles_pass_q<DT, true, LOCAL>(prow, qrow, V, c, sc, tile_sum, tlo, thi);
-    else tiles_pass_q<DT, false, LOCAL>(prow, qrow, V, c, sc, tile_sum, tlo, thi);
+    if (use_q) tiles_pass_q<DT, true>(prow, qrow, V, c, sc, tile_sum, tlo, thi);
+    else tiles_pass_q<DT, false>(prow, qrow, V, c, sc, tile_sum, tlo, thi);
 }
 
 // The token at `target` of the row's running sum, for the warp of the share that contains it: lane i of the warp
 // owns tiles [t0, t1) of the share with sum `mine` and inclusive running sum `incl` over the lanes, `base` is the mass
 // before the share.  Returns the token in every lane (-1 if the share holds no mass).
-template <int DT, bool COHERENT = false, bool LOCAL = false>
+template <int DT, bool COHERENT = false>
 __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow, int V, float c, const RowScale sc,
                                              bool use_q, const float* tile_sum, int t0, int t1, double mine, double incl,
                                              double base, double target, int lane)
@@ -368,7 +356,7 @@ __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow,
     }
     if (tile >= 0) {
         float r[8];
-        tile_resid<DT, LOCAL>(prow, qrow, tile * kTile + lane * 8, V, c, sc, use_q, r);
+        tile_resid<DT>(prow, qrow, tile * kTile + lane * 8, V, c, sc, use_q, r);
         double lane_sum = 0.0;
 #pragma unroll
         for (int e = 0; e < 8; ++e) lane_sum += static_cast<double>(r[e]);
@@ -399,17 +387,18 @@ __device__ __forceinline__ int pick_in_share(const void* prow, const void* qrow,
 // Inverse CDF of the residual (use_q) or of P (bonus / fallback) at uniform u.
 // Returns the token (same value in every thread) and, through *total_out, the total mass times the row's
 // common factor Z_p (only its sign is meaningful to the caller).
-template <int DT, bool LOCAL = false>
+template <int DT>
 __device__ int sample_row(const void* prow, const void* qrow, int V, float c, RowStat sp, RowStat sq, bool use_q,
                           float u, float* tile_sum, SampleShared* sh, double* total_out, const ClusterCtx cl)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ntiles = (V + kTile - 1) / kTile;
     // this CTA's share of the row: tiles [tlo, thi)
-    const int tlo = min(cl.rank * cl.tiles_per_rank, ntiles), thi = min(tlo + cl.tiles_per_rank, ntiles);
+    const int tiles_per_rank = (ntiles + cl.size - 1) / cl.size;
+    const int tlo = min(cl.rank * tiles_per_rank, ntiles), thi = min(tlo + tiles_per_rank, ntiles);
     const RowScale sc = row_scale(sp.E, sp.Z, sq.E, sq.Z, use_q);
 
-    tiles_pass<DT, LOCAL>(prow, qrow, V, c, sc, use_q, tile_sum, tlo, thi);
+    tiles_pass<DT>(prow, qrow, V, c, sc, use_q, tile_sum, tlo, thi);
     __syncthreads();
 
     // each lane of warp 0 owns a contiguous run of the CTA's tiles; tile sums are added in double, in order
@@ -444,7 +433,7 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
         if (owner_rank < 0) { owner_rank = last_mass; base = last_base; }      // u not below 1, or rounding
         int token = -1;
         if (owner_rank == cl.rank) {
-            token = pick_in_share<DT, false, LOCAL>(prow, qrow, V, c, sc, use_q, tile_sum, t0, t1, mine, incl, base, target, lane);
+            token = pick_in_share<DT>(prow, qrow, V, c, sc, use_q, tile_sum, t0, t1, mine, incl, base, target, lane);
         }
         if (lane == 0) sh->total = total;
         // the CTA that holds the token tells every CTA (with no mass anywhere, CTA 0 reports -1)
@@ -461,169 +450,6 @@ __device__ int sample_row(const void* prow, const void* qrow, int V, float c, Ro
     const int token = sh->token;
     __syncthreads();          // sh and tile_sum are reused by the next pass
     return token;
-}
-
-
-// Where the level loop finds a sequence's row-statistics partials and the rows of its pass.  The walk that follows
-// the row-statistics kernel reads both from global memory.
-template <int DT> struct GlobalRows {
-    static constexpr bool kLocal = false;
-    const WalkParams* p;
-    int b;
-    __device__ __forceinline__ const float2* partials(int model, int j) const
-    {
-        return p->partials + static_cast<size_t>(p->t.row_begin[model] + b * p->t.rows[model] + j) * p->parts;
-    }
-    // base of row j of `model`: element v of the row is at base + v * sizeof(element)
-    __device__ __forceinline__ const void* pass_row(int model, int j) const
-    {
-        constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
-        return static_cast<const char*>(p->t.logits[model]) + (static_cast<size_t>(b) * p->t.rows[model] + j) * p->V * ELEM;
-    }
-};
-
-// The level loop of one sequence (Section 3.1: checked bottom-up, by M_{n-1} first and M_1 last; per level
-// Algorithm 1's Verify with a break at the first failure, then the replacement or bonus token), run by every
-// CTA of the sequence's cluster in lockstep; only cluster rank 0 writes results.
-template <int DT, class Src>
-__device__ __forceinline__ void walk_levels(const WalkParams& p, const Src& src, const ClusterCtx cl, const int b, float* tile_sum)
-{
-    __shared__ int tok[kMaxK + 2];
-    __shared__ RowStat st_p[kMaxK + 1];
-    __shared__ RowStat st_q[kMaxK + 1];
-    __shared__ int sh_a, sh_bad;
-    __shared__ float g_zp[32], g_zq[32], g_u[32];       // logits at the block tokens, accept uniforms
-    __shared__ SampleShared sh_sample;
-
-    constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
-    const bool writer = cl.rank == 0;
-    const int tid = threadIdx.x;
-    const int L = p.n_levels;
-    const size_t row_bytes = static_cast<size_t>(p.V) * ELEM;
-    const double cd = static_cast<double>(p.c);
-
-    int stream_len = p.k[L - 1];
-    if (p.bottom_len) stream_len = max(0, min(stream_len, p.bottom_len[b]));
-    if (tid < p.k[L - 1]) tok[tid] = p.draft_tokens[static_cast<size_t>(b) * p.k[L - 1] + tid];
-    __syncthreads();
-
-    bool dead = false;
-    for (int l = L - 1; l >= 0; --l) {
-        const int kl = p.k[l];
-        const size_t lb = static_cast<size_t>(l) * p.B + b;
-        if (dead) {               // an unusable input below: this level reports -1 as well
-            if (writer && tid == 0) {
-                p.accepted_len[lb] = -1;
-                if (p.block_len) p.block_len[lb] = -1;
-                if (p.out_len) p.out_len[lb] = -1;
-            }
-            if (writer && p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
-            continue;
-        }
-        const int m = min(kl, stream_len);
-        const char* base_p = static_cast<const char*>(p.t.logits[l]) + static_cast<size_t>(b) * p.t.rows[l] * row_bytes;
-        const char* base_q = static_cast<const char*>(p.t.logits[l + 1]) + static_cast<size_t>(b) * p.t.rows[l + 1] * row_bytes;
-
-        // 1. normalisers of p rows 0..m and q rows 0..m-1; the last warp first requests the logits at the
-        // block tokens and the accept uniforms, so that those loads are in flight during the merges
-        if ((tid >> 5) == kWalkWarps - 1) {
-            const int j = tid & 31;
-            float zp = 0.0f, zq = 0.0f, uu = 0.0f;
-            if (j < m) {
-                const int x = tok[j];
-                if (x >= 0 && x < p.V) {
-                    zp = load_logit<DT>(base_p + j * row_bytes, x);
-                    zq = load_logit<DT>(base_q + j * row_bytes, x);
-                }
-                uu = p.uniforms[lb * (p.kmax + 1) + j];
-            }
-            g_zp[j] = zp;
-            g_zq[j] = zq;
-            g_u[j] = uu;
-        }
-        for (int r = tid >> 5; r < 2 * m + 1; r += kWalkWarps) {          // one warp per row
-            const bool is_q = r > m;
-            const int j = is_q ? r - (m + 1) : r;
-            const RowStat st = merge_partials(src.partials(is_q ? l + 1 : l, j), p.parts, tid & 31);
-            if ((tid & 31) == 0) (is_q ? st_q : st_p)[j] = st;
-        }
-        __syncthreads();
-
-        // 2. accept tests (warp 0; m <= 32)
-        if (tid < 32) {
-            bool rej = false, bad = false;
-            float pf = 0.0f, qf = 0.0f;
-            if (tid < m) {
-                const int x = tok[tid];
-                const RowStat sp = st_p[tid], sq = st_q[tid];
-                if (x < 0 || x >= p.V || !stat_ok(sp) || !stat_ok(sq)) {
-                    bad = true;
-                } else {
-                    const float zp = g_zp[tid], zq = g_zq[tid];
-                    const double P = exp2(static_cast<double>(zp) * cd - static_cast<double>(sp.E)) / sp.Z;
-                    const double Q = exp2(static_cast<double>(zq) * cd - static_cast<double>(sq.E)) / sq.Z;
-                    const double u = static_cast<double>(g_u[tid]);
-                    rej = !(u * Q <= P);
-                    pf = static_cast<float>(P);
-                    qf = static_cast<float>(Q);
-                }
-            }
-            if (writer && l == 0 && p.p_at && tid < kl) p.p_at[static_cast<size_t>(b) * kl + tid] = pf;
-            if (writer && l == 0 && p.q_at && tid < kl) p.q_at[static_cast<size_t>(b) * kl + tid] = qf;
-            const unsigned rej_mask = __ballot_sync(0xffffffffu, rej);
-            const unsigned bad_mask = __ballot_sync(0xffffffffu, bad);
-            const int first_rej = rej_mask ? (__ffs(rej_mask) - 1) : m;
-            const int first_bad = bad_mask ? (__ffs(bad_mask) - 1) : m + 1;
-            if (tid == 0) {
-                int isbad = first_bad < first_rej;
-                if (!isbad && first_rej == m && !stat_ok(st_p[m])) isbad = 1;     // bonus row unusable
-                sh_a = first_rej;
-                sh_bad = isbad;
-            }
-        }
-        __syncthreads();
-        const int a = sh_a;
-        if (sh_bad) {
-            dead = true;
-            if (writer && tid == 0) {
-                p.accepted_len[lb] = -1;
-                if (p.block_len) p.block_len[lb] = -1;
-                if (p.out_len) p.out_len[lb] = -1;
-                if (p.next_token) p.next_token[b] = -1;
-                if (p.device_status) atomicCAS(p.device_status, 0, static_cast<int>(POLYSPEC_ERR_BAD_INPUT_ON_DEVICE));
-            }
-            if (writer && p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
-            __syncthreads();
-            continue;
-        }
-
-        // 3. replacement (a < m) or bonus (a == m) token
-        const float u_s = p.uniforms[lb * (p.kmax + 1) + p.kmax];
-        const void* prow = src.pass_row(l, a);
-        const void* qrow = src.pass_row(l + 1, a);
-        bool use_q = a < m;
-        const RowStat sp = st_p[a];
-        const RowStat sq = use_q ? st_q[a] : sp;
-        double total = 0.0;
-        int next = sample_row<DT, Src::kLocal>(prow, qrow, p.V, p.c, sp, sq, use_q, u_s, tile_sum, &sh_sample, &total, cl);
-        if (use_q && !(total > 0.0)) {          // residual vanished in floating point: sample P instead
-            next = sample_row<DT, Src::kLocal>(prow, qrow, p.V, p.c, sp, sq, false, u_s, tile_sum, &sh_sample, &total, cl);
-        }
-
-        // 4. outputs and hand-off
-        if (writer && tid == 0) {
-            p.accepted_len[lb] = a;
-            if (p.block_len) p.block_len[lb] = m;
-            if (p.out_len) p.out_len[lb] = a + 1;
-            if (p.next_token) p.next_token[b] = next;
-        }
-        if (writer && p.out_tokens && tid <= p.kmax)
-            p.out_tokens[lb * (p.kmax + 1) + tid] = (tid < a) ? tok[tid] : (tid == a ? next : -1);
-        __syncthreads();
-        if (tid == 0) tok[a] = next;
-        stream_len = a + 1;
-        __syncthreads();
-    }
 }
 
 }  // namespace walkdev

@@ -30,6 +30,14 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* tile_sum = reinterpret_cast<float*>(smem_raw);
 
+    __shared__ int tok[kMaxK + 2];
+    __shared__ RowStat st_p[kMaxK + 1];
+    __shared__ RowStat st_q[kMaxK + 1];
+    __shared__ int sh_a, sh_bad;
+    __shared__ float g_zp[32], g_zq[32], g_u[32];       // logits at the block tokens, accept uniforms
+    __shared__ SampleShared sh_sample;
+
+    constexpr size_t ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
     // Launched with programmatic stream serialisation: the CTAs may be placed while the kernel before
     // (row statistics or the LM-head projection) is still finishing; nothing it wrote is touched before
     // this point.
@@ -44,13 +52,137 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
     ClusterCtx cl;
     cl.size = p.cluster;
     cl.rank = static_cast<int>(blockIdx.x) % p.cluster;
-    const int ntiles = (p.V + kTile - 1) / kTile;
-    cl.tiles_per_rank = (ntiles + cl.size - 1) / cl.size;
+    const bool writer = cl.rank == 0;
     const int b = static_cast<int>(blockIdx.x) / p.cluster;
-    GlobalRows<DT> src;
-    src.p = &p;
-    src.b = b;
-    walk_levels<DT>(p, src, cl, b, tile_sum);
+    const int tid = threadIdx.x;
+    const int L = p.n_levels;
+    const size_t row_bytes = static_cast<size_t>(p.V) * ELEM;
+    const double cd = static_cast<double>(p.c);
+
+    int stream_len = p.k[L - 1];
+    if (p.bottom_len) stream_len = max(0, min(stream_len, p.bottom_len[b]));
+    if (tid < p.k[L - 1]) tok[tid] = p.draft_tokens[static_cast<size_t>(b) * p.k[L - 1] + tid];
+    __syncthreads();
+
+    bool dead = false;
+    for (int l = L - 1; l >= 0; --l) {
+        const int kl = p.k[l];
+        const size_t lb = static_cast<size_t>(l) * p.B + b;
+        if (dead) {               // an unusable input below: this level reports -1 as well
+            if (writer && tid == 0) {
+                p.accepted_len[lb] = -1;
+                if (p.block_len) p.block_len[lb] = -1;
+                if (p.out_len) p.out_len[lb] = -1;
+            }
+            if (writer && p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
+            continue;
+        }
+        const int m = min(kl, stream_len);
+        const int grow_p = p.t.row_begin[l] + b * p.t.rows[l];
+        const int grow_q = p.t.row_begin[l + 1] + b * p.t.rows[l + 1];
+        const char* base_p = static_cast<const char*>(p.t.logits[l]) + static_cast<size_t>(b) * p.t.rows[l] * row_bytes;
+        const char* base_q = static_cast<const char*>(p.t.logits[l + 1]) + static_cast<size_t>(b) * p.t.rows[l + 1] * row_bytes;
+
+        // 1. normalisers of p rows 0..m and q rows 0..m-1; the last warp first requests the logits at the
+        // block tokens and the accept uniforms, so that those loads are in flight during the merges
+        if ((tid >> 5) == kWalkWarps - 1) {
+            const int j = tid & 31;
+            float zp = 0.0f, zq = 0.0f, uu = 0.0f;
+            if (j < m) {
+                const int x = tok[j];
+                if (x >= 0 && x < p.V) {
+                    zp = load_logit<DT>(base_p + j * row_bytes, x);
+                    zq = load_logit<DT>(base_q + j * row_bytes, x);
+                }
+                uu = p.uniforms[lb * (p.kmax + 1) + j];
+            }
+            g_zp[j] = zp;
+            g_zq[j] = zq;
+            g_u[j] = uu;
+        }
+        for (int r = tid >> 5; r < 2 * m + 1; r += kWalkWarps) {          // one warp per row
+            const bool is_q = r > m;
+            const int j = is_q ? r - (m + 1) : r;
+            const RowStat st = merge_partials(p.partials + static_cast<size_t>((is_q ? grow_q : grow_p) + j) * p.parts, p.parts, tid & 31);
+            if ((tid & 31) == 0) (is_q ? st_q : st_p)[j] = st;
+        }
+        __syncthreads();
+
+        // 2. accept tests (warp 0; m <= 32)
+        if (tid < 32) {
+            bool rej = false, bad = false;
+            float pf = 0.0f, qf = 0.0f;
+            if (tid < m) {
+                const int x = tok[tid];
+                const RowStat sp = st_p[tid], sq = st_q[tid];
+                if (x < 0 || x >= p.V || !stat_ok(sp) || !stat_ok(sq)) {
+                    bad = true;
+                } else {
+                    const float zp = g_zp[tid], zq = g_zq[tid];
+                    const double P = exp2(static_cast<double>(zp) * cd - static_cast<double>(sp.E)) / sp.Z;
+                    const double Q = exp2(static_cast<double>(zq) * cd - static_cast<double>(sq.E)) / sq.Z;
+                    const double u = static_cast<double>(g_u[tid]);
+                    rej = !(u * Q <= P);
+                    pf = static_cast<float>(P);
+                    qf = static_cast<float>(Q);
+                }
+            }
+            if (writer && l == 0 && p.p_at && tid < kl) p.p_at[static_cast<size_t>(b) * kl + tid] = pf;
+            if (writer && l == 0 && p.q_at && tid < kl) p.q_at[static_cast<size_t>(b) * kl + tid] = qf;
+            const unsigned rej_mask = __ballot_sync(0xffffffffu, rej);
+            const unsigned bad_mask = __ballot_sync(0xffffffffu, bad);
+            const int first_rej = rej_mask ? (__ffs(rej_mask) - 1) : m;
+            const int first_bad = bad_mask ? (__ffs(bad_mask) - 1) : m + 1;
+            if (tid == 0) {
+                int isbad = first_bad < first_rej;
+                if (!isbad && first_rej == m && !stat_ok(st_p[m])) isbad = 1;     // bonus row unusable
+                sh_a = first_rej;
+                sh_bad = isbad;
+            }
+        }
+        __syncthreads();
+        const int a = sh_a;
+        if (sh_bad) {
+            dead = true;
+            if (writer && tid == 0) {
+                p.accepted_len[lb] = -1;
+                if (p.block_len) p.block_len[lb] = -1;
+                if (p.out_len) p.out_len[lb] = -1;
+                if (p.next_token) p.next_token[b] = -1;
+                if (p.device_status) atomicCAS(p.device_status, 0, static_cast<int>(POLYSPEC_ERR_BAD_INPUT_ON_DEVICE));
+            }
+            if (writer && p.out_tokens && tid <= p.kmax) p.out_tokens[lb * (p.kmax + 1) + tid] = -1;
+            __syncthreads();
+            continue;
+        }
+
+        // 3. replacement (a < m) or bonus (a == m) token
+        const float u_s = p.uniforms[lb * (p.kmax + 1) + p.kmax];
+        const void* prow = base_p + a * row_bytes;
+        const void* qrow = base_q + a * row_bytes;
+        bool use_q = a < m;
+        const RowStat sp = st_p[a];
+        const RowStat sq = use_q ? st_q[a] : sp;
+        double total = 0.0;
+        int next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, use_q, u_s, tile_sum, &sh_sample, &total, cl);
+        if (use_q && !(total > 0.0)) {          // residual vanished in floating point: sample P instead
+            next = sample_row<DT>(prow, qrow, p.V, p.c, sp, sq, false, u_s, tile_sum, &sh_sample, &total, cl);
+        }
+
+        // 4. outputs and hand-off
+        if (writer && tid == 0) {
+            p.accepted_len[lb] = a;
+            if (p.block_len) p.block_len[lb] = m;
+            if (p.out_len) p.out_len[lb] = a + 1;
+            if (p.next_token) p.next_token[b] = next;
+        }
+        if (writer && p.out_tokens && tid <= p.kmax)
+            p.out_tokens[lb * (p.kmax + 1) + tid] = (tid < a) ? tok[tid] : (tid == a ? next : -1);
+        __syncthreads();
+        if (tid == 0) tok[a] = next;
+        stream_len = a + 1;
+        __syncthreads();
+    }
 }
 
 }  // namespace

@@ -216,29 +216,6 @@ def test_sharded_chain_calls_reject_bad_arguments_without_launching(lib):
     assert lib.polyspec_sharded_chain_handoff(4, k, 0, 256, fake, null, fake, fake, null, null, null) == binding.ERR_INVALID_ARG
 
 
-def test_launch_count_query_says_which_shapes_take_the_single_cluster_kernel():
-    """Host arithmetic of polyspec_verify_chain_launches: one kernel for a small batch whose rows fit the shared
-    memory of eight CTAs per sequence (the paper's batch size 1, Section 4.1), two otherwise."""
-    binding.load_library()
-    q = binding.polyspec_verify_chain_launches
-    bf, f32 = binding.BF16, binding.F32
-    assert q([4], [5, 4], 1, 32000, f32) == 1                          # two models, batch 1
-    assert q([9, 8], [10, 9, 8], 1, 32000, bf) == 1                    # three models, batch 1: 27 rows x 8 KiB per CTA
-    assert q([9, 9], [10, 10, 9], 1, 32000, bf) == 2                   # one row too many to stage
-    assert q([9, 8], [10, 9, 8], 16, 32000, bf) == 2                   # that many rows get longer segments: two launches
-    assert q([4], [5, 4], 16, 32000, f32) == 1
-    assert q([4], [5, 4], 17, 32000, f32) == 2                         # more sequences than the kernel takes
-    assert q([6, 6], [7, 7, 6], 1, 128256, bf) == 2                    # rows too long to stage
-    assert q([4, 6, 10], [5, 7, 11, 10], 1, 152064, bf) == 2
-    assert q([2, 3], [3, 4, 3], 3, 8, f32) == 1 and q([5], [6, 5], 2, 2048, bf) == 1      # rows of one segment
-    assert q([5], [6, 5], 2, 3000, f32) == 1 and q([2], [3, 2], 1, 151936, bf) == 1
-    with pytest.raises(binding.PolyspecError):
-        q([4], [4, 4], 1, 32000, f32)                                  # the verifier lacks its bonus row
-    lib = binding.load_library()
-    k, rows = (ctypes.c_int * 1)(4), (ctypes.c_int * 2)(5, 4)
-    assert lib.polyspec_verify_chain_launches(2, k, rows, 1, 32000, f32, None) == binding.ERR_INVALID_ARG
-
-
 def test_binding_raises_when_the_library_is_missing(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libpolyspec.so")
