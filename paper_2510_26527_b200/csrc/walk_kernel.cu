@@ -112,19 +112,27 @@ __global__ void __launch_bounds__(kWalkThreads, POLYSPEC_WALK_CTAS_PER_SM) walk_
         if (tid < 32) {
             bool rej = false, bad = false;
             float pf = 0.0f, qf = 0.0f;
+            const bool want_pq = writer && l == 0 && (p.p_at || p.q_at);      // the probabilities are a diagnostic output
             if (tid < m) {
                 const int x = tok[tid];
                 const RowStat sp = st_p[tid], sq = st_q[tid];
                 if (x < 0 || x >= p.V || !stat_ok(sp) || !stat_ok(sq)) {
                     bad = true;
                 } else {
+                    // u Q <= P with P = 2^xp / Z_p and Q = 2^xq / Z_q, taken as u Z_p 2^(xq - xp) <= Z_q: one
+                    // double-precision exponential and no division on the path every level waits for (the two
+                    // exponentials and divisions of the plain form are 1.5 us of dependent arithmetic).  Q = 0 or
+                    // u = 0 make the left side zero whatever the gap of the exponents: accepted.
                     const float zp = g_zp[tid], zq = g_zq[tid];
-                    const double P = exp2(static_cast<double>(zp) * cd - static_cast<double>(sp.E)) / sp.Z;
-                    const double Q = exp2(static_cast<double>(zq) * cd - static_cast<double>(sq.E)) / sq.Z;
+                    const double xp = static_cast<double>(zp) * cd - static_cast<double>(sp.E);
+                    const double xq = static_cast<double>(zq) * cd - static_cast<double>(sq.E);
                     const double u = static_cast<double>(g_u[tid]);
-                    rej = !(u * Q <= P);
-                    pf = static_cast<float>(P);
-                    qf = static_cast<float>(Q);
+                    const bool left_zero = zq == -INFINITY || !(u > 0.0);
+                    rej = !(left_zero || u * sp.Z * exp2(xq - xp) <= sq.Z);
+                    if (want_pq) {
+                        pf = static_cast<float>(exp2(xp) / sp.Z);
+                        qf = static_cast<float>(exp2(xq) / sq.Z);
+                    }
                 }
             }
             if (writer && l == 0 && p.p_at && tid < kl) p.p_at[static_cast<size_t>(b) * kl + tid] = pf;
