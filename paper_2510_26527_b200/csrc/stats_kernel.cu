@@ -219,18 +219,19 @@ constexpr size_t kStatsSmemBytes = static_cast<size_t>(kWarps) * kStages * (kChu
 
 StatsPlan plan_stats(long long total_rows, int V, polyspec_dtype dt)
 {
-    // A segment (one warp's work item) is a multiple of 2048 elements and at most 16 KiB.  Work items are dealt out to
-    // the 148 x kWarps warps in equal numbers, so the pass takes as long as the warp with the most items: among the
-    // admissible segment lengths take the one with the smallest (items per busiest warp) x (bytes per item + a fixed
-    // cost per item); on a tie the longer segment.  Few rows are thus cut finer (every SM still gets work), a mid-size
-    // problem gets a length that does not leave a fifth of the warps one item short (the three-level workload: 6144
-    // elements, 5.7 items per warp, instead of 8192, 4.3 per warp with a fifth item on a third of the warps), and a
-    // large one keeps 16 KiB.
+    // A segment (one warp's work item) is a whole number of 2 KiB chunks, at least 2048 elements and at most 16 KiB.
+    // Work items are dealt out to the 148 x kWarps warps in equal numbers, so the pass takes as long as the warp with
+    // the most items: among the admissible segment lengths take the one with the smallest (items per busiest warp) x
+    // (bytes per item + a fixed cost per item); on a tie the longer segment.  Few rows are thus cut finer (every SM
+    // still gets work), a mid-size problem gets a length that does not leave many warps one item short (the
+    // three-level workload: 7168 elements, 4.9 items per warp, instead of 8192, 4.3 per warp with a fifth item on a
+    // third of the warps), and a large one keeps 16 KiB.
     const long long elem = dt == POLYSPEC_BF16 ? 2 : 4;
     const long long seg_max = 16384LL / elem;
+    const long long step = kChunkBytes / elem;
     const long long warps = 148LL * kWarps;
     long long seg = 2048, best = -1;
-    for (long long cand = 2048; cand <= seg_max; cand += 2048) {
+    for (long long cand = 2048; cand <= seg_max; cand += step) {
         const long long items = total_rows * ((V + cand - 1) / cand);
         const long long per_warp = (items + warps - 1) / warps;
         const long long cost = per_warp * (std::min<long long>(cand, V) * elem + 512);
