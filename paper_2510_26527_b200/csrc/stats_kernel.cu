@@ -122,6 +122,8 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
         float best = -INFINITY;
         int best_at = 0x7fffffff;
         uint32_t abs_max = 0;              // largest |bits|: above 0x7f800000 means a NaN went by
+        PackedArgMax packed;               // 2-byte logits take the packed form instead
+        packed.init();
         const int seg_first = (item % p.parts) * p.seg;      // row index of the segment's first element
 
         for (uint32_t off = 0; off < bytes; off += kChunkBytes, ++done) {
@@ -162,6 +164,8 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
                 for (int u = 0; u < kVecPerLane; ++u)
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) s[u] += ex2f(__fmaf_rn(z[u][e], c, -E));
+            } else if (DT == POLYSPEC_BF16) {
+                packed.chunk(r, off / kChunkBytes);
             } else {
                 constexpr int ELEM = (DT == POLYSPEC_BF16) ? 2 : 4;
 #pragma unroll
@@ -185,6 +189,13 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
         }
 
         if (MODE == 1) {
+            if (DT == POLYSPEC_BF16) {
+                bool nan;
+                packed.finish(lane, &best, &best_at, &nan);
+                // a lane that saw nothing but -inf keeps the "no index" mark, like the scalar form
+                best_at = (best == -INFINITY) ? 0x7fffffff : seg_first + best_at;
+                abs_max = nan ? 0x7fc00000u : 0u;
+            }
             // lanes -> warp: the larger value wins, equal values go to the lower index
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {

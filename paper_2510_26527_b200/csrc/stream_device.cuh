@@ -138,5 +138,49 @@ template <> struct Elems<POLYSPEC_F32> {
     }
 };
 
+// Arg max of 2-byte logits on the packed words: the running maximum of the even and of the odd elements a lane has
+// seen, two per instruction, NaN sticking once met (max.NaN); where a half's maximum moved is kept, branch-free, as
+// the word's number inside its chunk (ppos) and, once per chunk, the chunk's number (pchunk), both packed like the
+// maxima.  A value equal to the running maximum does not move it, so what is kept is the first occurrence.
+struct PackedArgMax {
+    uint32_t pm, ppos, pchunk;
+    __device__ __forceinline__ void init() { pm = 0xff80ff80u; ppos = 0; pchunk = 0; }
+    template <uint32_t J> __device__ __forceinline__ void word(uint32_t w)
+    {
+        uint32_t nm, moved;
+        asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(nm) : "r"(pm), "r"(w));
+        asm("set.neu.u32.bf16x2 %0, %1, %2;" : "=r"(moved) : "r"(nm), "r"(pm));        // 0xffff per half that moved
+        ppos = (ppos & ~moved) | (((J << 16) | J) & moved);
+        pm = nm;
+    }
+    // the four vectors (sixteen words) a lane holds of one chunk; `chunk` is the chunk's number in the segment
+    __device__ __forceinline__ void chunk(const uint4 (&r)[kVecPerLane], uint32_t chunk_no)
+    {
+        const uint32_t before = pm;
+        word<0>(r[0].x); word<1>(r[0].y); word<2>(r[0].z); word<3>(r[0].w);
+        word<4>(r[1].x); word<5>(r[1].y); word<6>(r[1].z); word<7>(r[1].w);
+        word<8>(r[2].x); word<9>(r[2].y); word<10>(r[2].z); word<11>(r[2].w);
+        word<12>(r[3].x); word<13>(r[3].y); word<14>(r[3].z); word<15>(r[3].w);
+        uint32_t moved;
+        asm("set.neu.u32.bf16x2 %0, %1, %2;" : "=r"(moved) : "r"(pm), "r"(before));
+        pchunk = (pchunk & ~moved) | (((chunk_no << 16) | chunk_no) & moved);
+    }
+    // The lane's best (value, element index inside the segment) and whether it met a NaN.
+    __device__ __forceinline__ void finish(int lane, float* best, int* at, bool* nan) const
+    {
+        const uint32_t lo = pm & 0xffffu, hi = pm >> 16;
+        *nan = (lo & 0x7fffu) > 0x7f80u || (hi & 0x7fffu) > 0x7f80u;
+        const float vlo = __uint_as_float(lo << 16), vhi = __uint_as_float(hi << 16);
+        // word j of chunk c is word (j & 3) of the lane's vector (j >> 2), which is vector (j >> 2) * 32 + lane of the chunk
+        auto element = [&](uint32_t c, uint32_t j, uint32_t half) {
+            return static_cast<int>(c * (kChunkBytes / 2) + ((j >> 2) * 32 + lane) * 8 + (j & 3) * 2 + half);
+        };
+        const int alo = element(pchunk & 0xffffu, ppos & 0xffffu, 0), ahi = element(pchunk >> 16, ppos >> 16, 1);
+        const bool take_hi = vhi > vlo || (vhi == vlo && ahi < alo);
+        *best = take_hi ? vhi : vlo;
+        *at = take_hi ? ahi : alo;
+    }
+};
+
 }  // namespace streamdev
 }  // namespace polyspec
