@@ -95,6 +95,45 @@ def test_unusable_inputs(oracle):
                 assert (got[key][0, b] == ora[key][0, b]).all(), (key, b)
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_planted_maxima_at_every_word_position_chunk_and_segment(dtype):
+    """The arg max of 2-byte logits is kept on packed words with its position recorded per half, per word and per
+    chunk: a unique maximum planted at every kind of position (both halves of every word of a lane's four vectors,
+    first and later chunks, first and later segments, the ragged end), the same value planted twice (the first
+    must win), +0 against -0, and a maximum equal to the largest finite value.  Row 0's arg max is what the rule
+    emits after a mismatch at position 0, so it is read off next to torch's own arg max."""
+    V = 3 * 8192 + 1032                                    # three whole segments and a ragged fourth (2-byte logits)
+    idx = sorted(set([0, 1, 2, 7, 8, 255, 256, 257, 511, 1023, 1024, 1025, 2047, 2048, 4095, 4096, 8191, 8192, 8193,
+                      8192 + 1024 + 37, 2 * 8192 - 1, 2 * 8192, 3 * 8192 + 1031, V - 1, V - 8]
+                     + [(j * 2 + h) + 8 * (u * 32 + lane) + 1024 * c for j in range(4) for h in (0, 1)
+                        for u in range(4) for lane in (0, 5, 31) for c in (0, 3, 7)]))
+    idx = [i for i in idx if i < V]
+    B = len(idx) + 6
+    g = torch.Generator(device=DEV).manual_seed(12)
+    lp = (torch.randn((B, 2, V), generator=g, device=DEV) * 2).clamp(-8, 8)
+    for b, i in enumerate(idx):
+        lp[b, 0, i] = 16.0                                  # a unique maximum
+    n = len(idx)
+    lp[n + 0, 0, 4097] = 16.0; lp[n + 0, 0, 20001] = 16.0   # the same value twice: the first wins
+    lp[n + 1, 0, 9] = 16.0; lp[n + 1, 0, 8] = 16.0          # twice inside one word
+    lp[n + 2, 0] = -1.0; lp[n + 2, 0, 300] = -0.0; lp[n + 2, 0, 77] = 0.0      # +0 and -0 compare equal: index 77
+    lp[n + 3, 0] = -1.0; lp[n + 3, 0, 77] = -0.0; lp[n + 3, 0, 300] = 0.0      # ... and the other way round: still 77
+    lp[n + 4, 0, 12345] = 3.3895e38                         # the largest finite 2-byte value, not +inf
+    lp[n + 5, 0] = float("-inf"); lp[n + 5, 0, V - 3] = -1e30
+    lp = lp.to(dtype).contiguous()
+    want = lp[:, 0].float().argmax(-1)                      # torch returns the first maximal index too
+    assert want[n + 2].item() == 77 and want[n + 3].item() == 77 and want[n + 0].item() == 4097
+    draft = ((want + 1) % V).to(torch.int32).reshape(B, 1).contiguous()         # never the arg max: a = 0 everywhere
+    got = _run([lp, None], [1], draft)
+    assert got["device_status"][0] == 0
+    assert (got["accepted_len"][0] == 0).all()
+    assert (got["out_tokens"][0, :, 0] == want.cpu().numpy()).all(), np.argwhere(got["out_tokens"][0, :, 0] != want.cpu().numpy())[:8]
+    # and with the arg max drafted, everything is accepted and the bonus row's arg max follows
+    got = _run([lp, None], [1], want.to(torch.int32).reshape(B, 1).contiguous())
+    assert (got["accepted_len"][0] == 1).all()
+    assert (got["out_tokens"][0, :, 1] == lp[:, 1].float().argmax(-1).cpu().numpy()).all()
+
+
 @pytest.mark.parametrize("name,B,V,sigma", [("cfg2", 24, 4096, None), ("cfg3", 16, 10000, None), ("cfg5", 12, 8200, 0.25)])
 def test_chain_greedy_reduced(oracle, name, B, V, sigma):
     spec = synth.scaled(synth.config(name, sigma=sigma), B=B, V=V)
