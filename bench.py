@@ -140,8 +140,15 @@ def verified_tokens(block_len) -> int:
 
 
 def spread(ms):
-    """mean / median / min of a list of per-step times in milliseconds."""
-    return {"mean": float(np.mean(ms)), "median": float(np.median(ms)), "min": float(np.min(ms))}
+    """mean / median / min of a list of per-step times in milliseconds, and the means of the first and the last tenth
+    of the steps: a board that streams for tenths of a second may slow down under its power management, and the two
+    tenths show whether this run met that."""
+    out = {"mean": float(np.mean(ms)), "median": float(np.median(ms)), "min": float(np.min(ms))}
+    n = len(ms) // 10
+    if n >= 5:
+        out["first_tenth_mean"] = float(np.mean(ms[:n]))
+        out["last_tenth_mean"] = float(np.mean(ms[-n:]))
+    return out
 
 
 # ----------------------------------------------------------------------------------------- parity of the timed batch
