@@ -5,4 +5,4 @@ speculative decoding as hand-written CUDA kernels for sm_100a behind a C ABI.
 only), ``synth`` the seeded input generators, ``buildlib`` the nvcc build step.
 Nothing is loaded at import time; the binding raises if the CUDA library is missing.
 """
-__version__ = "0.3.0"      # polyspec_version() == 300
+__version__ = "0.3.1"      # polyspec_version() == 310

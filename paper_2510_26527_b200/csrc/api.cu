@@ -223,7 +223,7 @@ const char* polyspec_status_string(polyspec_status s)
     return "unknown status";
 }
 
-int polyspec_version(void) { return 300; }      // 0.3.0: single-launch chain, staged verification added to the ABI
+int polyspec_version(void) { return 310; }      // 0.3.1: staged verification and the second insertion condition in the ABI
 
 const char* polyspec_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 

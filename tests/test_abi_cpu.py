@@ -221,3 +221,9 @@ def test_binding_raises_when_the_library_is_missing(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libpolyspec.so")
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         binding.load_library()
+
+
+def test_package_and_library_versions_agree():
+    import paper_2510_26527_b200 as pkg
+    major, minor, patch = (int(x) for x in pkg.__version__.split("."))
+    assert binding.load_library().polyspec_version() == major * 1000 + minor * 100 + patch * 10
