@@ -78,3 +78,38 @@ def test_copy_wait_that_runs_out_reports_timeout_and_leaves_the_device_usable(or
     assert not bad and counts["exact"] == 8 * 2
     with pytest.raises(binding.PolyspecError):
         call.row_stats_wait_limit(0)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_the_largest_vocabulary_the_library_takes(oracle, dtype):
+    """V = 8192 tiles of 256 entries, the most the sampling pass keeps tile sums for: three models on two sequences
+    against the oracle (both rules), the token drawn from the far end of a row included; eight entries more are
+    refused before anything is launched."""
+    V, B, k = 8192 * 256, 2, [2, 3]
+    g = torch.Generator(device=DEV).manual_seed(91)
+    rows = [k[0] + 1, k[1] + 1, k[1]]
+    base = torch.randn((B, 4, V), generator=g, device=DEV) * 3.0
+    models = []
+    for i, r in enumerate(rows):
+        m = base[:, :r] if i == 0 else base[:, :r] + torch.randn((B, r, V), generator=g, device=DEV) * 0.7
+        models.append(m.to(dtype).contiguous())
+    del base
+    q = torch.softmax(models[-1].float(), dim=-1)
+    drafts = torch.multinomial(q.reshape(-1, V), 1, generator=g).reshape(B, k[1]).to(torch.int32).contiguous()
+    del q
+    u = torch.from_numpy(synth.philox_uniforms(92, 2, B, max(k) + 1)).to(DEV)
+    u[:, 1, max(k)] = 0.99999994                 # sequence 1 samples at the very end of the running sum at both levels
+    out = _np(binding.polyspec_verify_chain(models, k, drafts, u, 1.0))
+    ora = oracle.verify_chain([m.cpu() for m in models], k, drafts.cpu(), u.cpu(), 1.0, threads=8)
+    counts, bad = H.compare_chain(out, ora)
+    assert not bad, bad[:2]
+    assert out["device_status"][0] == 0
+    assert out["out_tokens"][:, 1].max() > V - V // 50          # the late uniform did reach the far end of a row
+    got = binding.polyspec_verify_chain_greedy(models, k, drafts)
+    torch.cuda.synchronize()
+    gra = oracle.verify_chain_greedy([m.cpu() for m in models], k, drafts.cpu(), threads=8)
+    for key in KEYS:
+        assert (got[key].cpu().numpy() == gra[key]).all(), key
+    with pytest.raises(binding.PolyspecError) as e:
+        binding.polyspec_verify_chain_workspace(k, rows, B, V + 8, binding._dt(models[0]))
+    assert e.value.status == binding.ERR_UNSUPPORTED
