@@ -80,6 +80,26 @@ def copy_probe_gbs(dev, nbytes=1 << 30, iters=20):
     return 2.0 * nbytes * iters / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
 
+def copy_probe_sustained_gbs(dev, nbytes=1 << 30, seconds=0.5):
+    """The same copy kept up for about as long as the timed region: (bandwidth over its first tenth, over its last tenth).
+
+    A board that streams for tenths of a second settles at a lower bandwidth than it shows in a burst; a kernel timed
+    over a thousand steps is mostly in that state, and this is the copy in the same state."""
+    src = torch.empty(nbytes, dtype=torch.uint8, device=dev).fill_(1)
+    dst = torch.empty_like(src)
+    iters = max(100, int(seconds / (2.0 * nbytes / 6.0e12)) // 10 * 10)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(11)]
+    torch.cuda.synchronize()
+    for seg in range(10):
+        marks[seg].record()
+        for _ in range(iters // 10):
+            dst.copy_(src)
+    marks[10].record()
+    torch.cuda.synchronize()
+    per_seg = 2.0 * nbytes * (iters // 10) / 1e9
+    return per_seg / (marks[0].elapsed_time(marks[1]) * 1e-3), per_seg / (marks[9].elapsed_time(marks[10]) * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -531,7 +551,10 @@ def measure_chain(env, args, spec, steps, warmup, headline):
         rec["l2_cold"] = cold
     if headline:
         live_copy = copy_probe_gbs(dev)
-        rec["roofline"].update({"this_gpu_copy_gbs": live_copy, "frac_of_this_gpu_copy": achieved / live_copy})
+        copy_first, copy_last = copy_probe_sustained_gbs(dev)
+        rec["roofline"].update({"this_gpu_copy_gbs": live_copy, "frac_of_this_gpu_copy": achieved / live_copy,
+                                "this_gpu_copy_sustained_gbs": {"first_tenth": copy_first, "last_tenth": copy_last},
+                                "frac_of_this_gpu_sustained_copy": achieved / copy_last})
         rec["e2e"] = {"value": tokens_all * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                       "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
                       "matches_device_path": same}

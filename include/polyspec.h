@@ -40,10 +40,11 @@
  *     holding NaN / +inf or no finite logit) never trap: the affected sequence gets
  *     accepted_len = next_token = -1 (and -1 in every later level of a chain) and
  *     *device_status is set to POLYSPEC_ERR_BAD_INPUT_ON_DEVICE.
- *   - No kernel polls memory without a limit.  Should a wait on a copy or on the tensor core
- *     ever run out, *device_status becomes POLYSPEC_ERR_TIMEOUT, the outputs of that call are
- *     undefined, and the kernels still return.  The only other waits are hardware barriers
- *     (block, cluster, grid dependency) that every participant reaches unconditionally.
+ *   - No kernel polls memory without a limit.  The kernels of the logits path wait on nothing but
+ *     hardware barriers (block, cluster, grid dependency) that every participant reaches
+ *     unconditionally.  The LM-head projection waits on its TMA copies and on the tensor core with
+ *     bounded polls: should one ever run out, *device_status becomes POLYSPEC_ERR_TIMEOUT, the
+ *     outputs of that call are undefined, and the kernel still returns.
  */
 #ifndef POLYSPEC_H
 #define POLYSPEC_H
@@ -149,18 +150,6 @@ polyspec_status polyspec_chain_walk(
     const int32_t* draft_tokens, const float* uniforms, int B, int V, polyspec_dtype dt, float temperature,
     int32_t* accepted_len, int32_t* block_len, int32_t* out_tokens, int32_t* out_len,
     int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream);
-
-/*
- * polyspec_chain_row_stats_wait_limit -- polyspec_chain_row_stats with the number of looks a warp may take at
- * the barrier of one of its copies set by the caller (the library's own wait is 2^20 suspending polls).  A diagnostic
- * for the give-up path described in the conventions above: with a limit too small for a copy to land, warps record
- * POLYSPEC_ERR_TIMEOUT in *device_status, still wait (with the full limit) for the copies they have in flight, and
- * return; the workspace contents are then undefined and the device stays usable.  wait_limit >= 1.
- */
-polyspec_status polyspec_chain_row_stats_wait_limit(
-    const polyspec_model_logits* models /* host */, int n_models, const int* k /* host */, int B, int V,
-    polyspec_dtype dt, float temperature, unsigned int wait_limit, int32_t* device_status, void* workspace,
-    size_t workspace_bytes, void* cuda_stream);
 
 /*
  * polyspec_verify_chain_host -- the same call for a caller whose buffers live in HOST

@@ -36,7 +36,6 @@ EXPORTS = (
     "polyspec_sharded_level_pick",
     "polyspec_sharded_chain_sizes", "polyspec_sharded_chain_stats", "polyspec_sharded_chain_gather",
     "polyspec_sharded_chain_decide", "polyspec_sharded_chain_pick", "polyspec_sharded_chain_handoff",
-    "polyspec_chain_row_stats_wait_limit",
     "polyspec_staged_init", "polyspec_staged_round_begin", "polyspec_staged_accumulate", "polyspec_staged_commit",
 )
 
@@ -104,8 +103,6 @@ def load_library() -> ctypes.CDLL:
     lib.polyspec_chain_row_stats.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, i32p, vp, sz, vp]
     lib.polyspec_chain_walk.restype = ci
     lib.polyspec_chain_walk.argtypes = lib.polyspec_verify_chain.argtypes
-    lib.polyspec_chain_row_stats_wait_limit.restype = ci
-    lib.polyspec_chain_row_stats_wait_limit.argtypes = [ctypes.POINTER(ModelLogits), ci, cip, ci, ci, ci, cf, ctypes.c_uint, i32p, vp, sz, vp]
     lib.polyspec_verify_chain_host_workspace.restype = ci
     lib.polyspec_verify_chain_host_workspace.argtypes = [ci, cip, cip, ci, ci, ci, szp]
     lib.polyspec_verify_chain_host.restype = ci
@@ -389,12 +386,6 @@ class ChainCall:
         _check(self.lib.polyspec_chain_row_stats(self._arr, self.n, self._k, self.B, self.V, self.dt, self.temperature,
                                                  _ptr(self.device_status), _ptr(self.workspace), self.workspace.numel(), _stream(self.stream)),
                "polyspec_chain_row_stats")
-
-    def row_stats_wait_limit(self, wait_limit: int):
-        _check(self.lib.polyspec_chain_row_stats_wait_limit(self._arr, self.n, self._k, self.B, self.V, self.dt, self.temperature,
-                                                            int(wait_limit), _ptr(self.device_status), _ptr(self.workspace),
-                                                            self.workspace.numel(), _stream(self.stream)),
-               "polyspec_chain_row_stats_wait_limit")
 
     def walk(self):
         _check(self.lib.polyspec_chain_walk(self._arr, self.n, self._k, _ptr(self.draft_tokens), _ptr(self.uniforms),

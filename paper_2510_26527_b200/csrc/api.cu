@@ -109,8 +109,6 @@ polyspec_status prepare_chain(const ChainArgs& a, StatsPlan* pl, StatsParams* sp
     sp->n_items = static_cast<int>(pl->n_items);
     sp->c = static_cast<float>(kLog2e / static_cast<double>(a.temperature));
     sp->partials = static_cast<float2*>(a.workspace);
-    sp->status = a.device_status;
-    sp->spin_limit = a.spin_limit;
     return POLYSPEC_OK;
 }
 
@@ -328,17 +326,6 @@ polyspec_status polyspec_verify_chain(
     return run_chain(a);
 }
 
-polyspec_status polyspec_chain_row_stats_wait_limit(
-    const polyspec_model_logits* models, int n_models, const int* k, int B, int V, polyspec_dtype dt,
-    float temperature, unsigned int wait_limit, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
-{
-    if (!models || !k || n_models < 2 || n_models > kMaxModels || wait_limit == 0) return POLYSPEC_ERR_INVALID_ARG;
-    ChainArgs a = chain_args(models, n_models, k, B, V, dt, temperature, workspace, workspace_bytes, cuda_stream);
-    a.device_status = device_status;
-    a.spin_limit = wait_limit;
-    return run_stats(a);
-}
-
 polyspec_status polyspec_chain_row_stats(
     const polyspec_model_logits* models, int n_models, const int* k, int B, int V, polyspec_dtype dt,
     float temperature, int32_t* device_status, void* workspace, size_t workspace_bytes, void* cuda_stream)
@@ -457,8 +444,6 @@ polyspec_status polyspec_verify_chain_greedy(
     sp.n_items = static_cast<int>(pl.n_items);
     sp.c = 1.0f;
     sp.partials = static_cast<float2*>(workspace);
-    sp.status = device_status;
-    sp.spin_limit = 0;
     if (cuda_failed(launch_stats(dt, sp, s, /*argmax=*/true))) return POLYSPEC_ERR_CUDA;
 
     WalkParams wp;

@@ -45,8 +45,6 @@ struct StatsParams {
     int n_items;
     float c;
     float2* partials;   // [total rows, parts]
-    int32_t* status;    // [1] or nullptr: receives POLYSPEC_ERR_TIMEOUT if a bounded wait expires
-    uint32_t spin_limit;   // 0: the default wait (2^20 suspending try_waits); otherwise that many non-suspending looks
 };
 
 // Decision + sampling pass: one CTA walks one sequence up the chain.

@@ -475,8 +475,6 @@ polyspec_status run_stats_and_merge(const void* const* logits, const int* rows, 
     sp.n_items = static_cast<int>(sz.plan.n_items);
     sp.c = p.c;
     sp.partials = const_cast<float2*>(p.partials);
-    sp.status = device_status;
-    sp.spin_limit = 0;
     if (cuda_failed(launch_stats(dt, sp, stream))) return POLYSPEC_ERR_CUDA;
     const unsigned blocks = static_cast<unsigned>((sz.rec_rows + 7) / 8);
     shard_merge_kernel<<<blocks, 256, 0, stream>>>(p.partials, p.parts, sz.rec_rows, static_cast<unsigned char*>(record));

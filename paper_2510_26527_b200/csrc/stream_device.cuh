@@ -1,6 +1,5 @@
-// Device helpers of the kernels that stream logits rows through per-warp shared-memory rings with 1-D bulk
-// TMA copies (the row-statistics kernel and the single-launch chain kernel): mbarrier and bulk-copy wrappers
-// with bounded waits, the unpacking of 16-byte vectors, exact power-of-two rescaling.
+// Device helpers of the row-statistics kernel: the streaming load, the unpacking of 16-byte vectors, exact
+// power-of-two rescaling, the packed arg max of 2-byte logits.
 #pragma once
 
 #include "polyspec_kernels.cuh"
@@ -8,75 +7,21 @@
 namespace polyspec {
 namespace streamdev {
 
-constexpr int kChunkBytes = 2048;                 // one bulk copy = one warp-wide sweep of 4 vectors per lane
-#ifndef POLYSPEC_STATS_STAGES
-#define POLYSPEC_STATS_STAGES 2
-#endif
+constexpr int kChunkBytes = 2048;                 // one warp-wide sweep of 4 vectors per lane
 #ifndef POLYSPEC_STATS_WARPS
 #define POLYSPEC_STATS_WARPS 32
 #endif
-// Measured on the four-level workload: 32 warps x 2 stages 402 us, 28 x 3 410 us, 24 x 4 419 us; warp counts
-// that are not multiples of four (one per scheduler) lose 5 %.
-constexpr int kStages = POLYSPEC_STATS_STAGES;    // per-warp ring depth
+// Warp counts that are not multiples of four (one per scheduler) lose 5 %.
 constexpr int kWarps = POLYSPEC_STATS_WARPS;
 constexpr int kStatsThreads = kWarps * 32;
 constexpr int kVecPerLane = kChunkBytes / 16 / 32;   // 4
-constexpr uint32_t kSpinLimit = 1u << 20;         // try_wait attempts before giving up
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// One look at the barrier without suspending the thread (try_wait may park it for a while before it answers).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// At most `limit` non-suspending looks: the caller-chosen limit of the diagnostic entry point.
-__device__ __forceinline__ bool wait_polls(uint32_t bar, uint32_t parity, uint32_t limit)
-{
-    for (uint32_t i = 0; i < limit; ++i)
-        if (mbar_test_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = kSpinLimit)
-{
-    for (uint32_t i = 0; i < limit; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-
-__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
+// A 16-byte vector of a row that is read once: through the read-only path, not kept in L1.
+__device__ __forceinline__ uint4 ld_stream(const void* p)
 {
     uint4 r;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
     return r;
 }
 

@@ -1,5 +1,5 @@
 """Edge cases of the chain call on the GPU that the parity file does not reach: unusable input that only an upper
-level meets, a residual that vanishes in floating point, and the give-up path of the row-statistics kernel."""
+level meets, a residual that vanishes in floating point, the largest vocabulary."""
 import numpy as np
 import pytest
 import torch
@@ -58,26 +58,6 @@ def test_residual_that_vanishes_falls_back_to_the_verifier_row(oracle):
         ora = oracle.verify_level(lp.cpu(), lq.cpu(), tok.cpu(), u.cpu(), 1.0)
         assert (ora["fallback"] == 1).all() and (out["accepted_len"] == 0).all()
         assert (out["next_token"] == ora["next_token"]).all(), (Vv, out["next_token"], ora["next_token"])
-
-
-def test_copy_wait_that_runs_out_reports_timeout_and_leaves_the_device_usable(oracle):
-    """The give-up path of the row-statistics kernel, in the safe form: the wait for a copy is given a single look, which a
-    copy from HBM cannot meet; the warps record POLYSPEC_ERR_TIMEOUT, still wait (full limit) for the copies they
-    have in flight, and return.  The next ordinary call on the same device and workspace is exact."""
-    spec = synth.scaled(synth.config("cfg3"), B=8, V=65536)
-    d = synth.make_chain(spec, seed=17, device=DEV)
-    call = binding.ChainCall(d["models"], d["k"], d["draft_tokens"], d["uniforms"], d["temperature"])
-    call.row_stats_wait_limit(1)
-    torch.cuda.synchronize()
-    assert int(call.device_status.item()) == binding.ERR_TIMEOUT
-    call.device_status.zero_()
-    call.row_stats()
-    out = _np(call.walk())
-    assert out["device_status"][0] == 0
-    counts, bad = H.compare_chain(out, _oracle(oracle, d))
-    assert not bad and counts["exact"] == 8 * 2
-    with pytest.raises(binding.PolyspecError):
-        call.row_stats_wait_limit(0)
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
