@@ -45,7 +45,7 @@ TIE_BAND = 1e-6
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the kernel that streams the logits, from the
 # ncu capture summarised under profiles/ (bytes per logits byte processed, measured on a smaller case of
 # the same kernel and scaled by the bytes one launch processes).  None once the kernel has changed since.
-STATS_TRAFFIC_PER_LOGIT_BYTE = 1.0130     # profiles/stats_kernel_bf16_cfg3_ncu_full.md: (328.350 + 4.250) MB moved for 328.340 MB of logits
+STATS_TRAFFIC_PER_LOGIT_BYTE = 1.0116     # profiles/stats_kernel_bf16_cfg3_ncu_full.md: (328.350 + 3.80) MB moved for 328.340 MB of logits
 # the same counters per launch of the LM-head kernel on the fused workload
 # (profiles/lmhead_kernel_cfg4_ncu.md: 402.98 MB read + 53.81 MB written)
 LMHEAD_TRAFFIC_BYTES = 456789504
