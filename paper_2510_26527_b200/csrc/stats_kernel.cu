@@ -48,6 +48,8 @@ __global__ void __launch_bounds__(kStatsThreads, 1) stats_kernel(const StatsPara
     using EL = Elems<DT>;
     constexpr int EPV = EL::per_vec;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // nothing the stream's earlier work wrote is read before this point (see launch_stats)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // consecutive items go to different CTAs: small problems still spread over every SM
     const int stride = gridDim.x * kWarps;
@@ -238,14 +240,25 @@ cudaError_t launch_stats(polyspec_dtype dt, const StatsParams& p, cudaStream_t s
     sm_count = g_sm_count[dev];
     }
     const int grid = p.n_items < sm_count ? p.n_items : sm_count;   // one CTA per SM
+    // Programmatic stream serialisation: the launch may be set up while the kernel before it on the stream (whatever
+    // wrote the logits, or the walk of the call before) is still draining; griddepcontrol.wait at the top of the kernel
+    // holds every read until that kernel has completed.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(kStatsThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (dt == POLYSPEC_BF16) {
-        if (argmax) stats_kernel<POLYSPEC_BF16, 1><<<grid, kStatsThreads, 0, stream>>>(p);
-        else stats_kernel<POLYSPEC_BF16, 0><<<grid, kStatsThreads, 0, stream>>>(p);
-    } else {
-        if (argmax) stats_kernel<POLYSPEC_F32, 1><<<grid, kStatsThreads, 0, stream>>>(p);
-        else stats_kernel<POLYSPEC_F32, 0><<<grid, kStatsThreads, 0, stream>>>(p);
+        if (argmax) return cudaLaunchKernelEx(&cfg, stats_kernel<POLYSPEC_BF16, 1>, p);
+        return cudaLaunchKernelEx(&cfg, stats_kernel<POLYSPEC_BF16, 0>, p);
     }
-    return cudaGetLastError();
+    if (argmax) return cudaLaunchKernelEx(&cfg, stats_kernel<POLYSPEC_F32, 1>, p);
+    return cudaLaunchKernelEx(&cfg, stats_kernel<POLYSPEC_F32, 0>, p);
 }
 
 }  // namespace polyspec
