@@ -468,6 +468,34 @@ def measure_chain(env, args, spec, steps, warmup, headline):
     # the same steps as single C-ABI calls, no event inside a step
     whole_ms, whole_steps, _, _ = timed_region(env, [call], lambda c: [("call", c.launch)], steps, False)
 
+    # ---- inputs that fit in L2 (the batch-1 workloads): also as a replayed CUDA graph of ten calls, which is how a
+    # decode loop would issue a step this short, and which takes the host's launch cost out of the figure
+    graph = None
+    if fits_l2 and world == 1:
+        side = torch.cuda.Stream(device=dev)
+        gcall = binding.ChainCall(data["models"], data["k"], data["draft_tokens"], data["uniforms"], data["temperature"],
+                                  stream=side.cuda_stream)
+        with torch.cuda.stream(side):
+            gcall.launch()
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(10):
+                    gcall.launch()
+            for _ in range(5):
+                g.replay()
+            side.synchronize()
+            reps = max(20, steps // 10)
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+            marks[0].record(side)
+            for i in range(reps):
+                g.replay()
+                marks[i + 1].record(side)
+            side.synchronize()
+        same_graph = all(torch.equal(gcall.out[n], call.out[n]) for n in ("accepted_len", "block_len", "out_tokens", "out_len"))
+        graph = {"calls_per_graph": 10, "replays": reps, "matches_plain_calls": bool(same_graph),
+                 "us_per_call": spread([100.0 * marks[i].elapsed_time(marks[i + 1]) for i in range(reps)])}
+
     # ---- inputs that fit in L2: also L2-cold, rotating through >= 256 MB of distinct instances of the workload
     cold = None
     if fits_l2 and world == 1:
@@ -549,6 +577,8 @@ def measure_chain(env, args, spec, steps, warmup, headline):
     }
     if cold is not None:
         rec["l2_cold"] = cold
+    if graph is not None:
+        rec["cuda_graph"] = graph
     if headline:
         live_copy = copy_probe_gbs(dev)
         copy_first, copy_last = copy_probe_sustained_gbs(dev)
